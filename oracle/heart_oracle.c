@@ -1,0 +1,465 @@
+/*
+ * heart_oracle.c -- CPU oracle for the HEART sparse-attention hot path.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, obviously-correct
+ * statement of what the hot path computes.  Only the test-suite, the smoke
+ * check and the benchmark's CPU-baseline leg may build or call it; the product
+ * (the CUDA library) shares no code with it and never calls it.
+ *
+ * Everything is fp64: bf16 inputs are widened exactly, every sum is a plain
+ * left-to-right fp64 loop, softmax is two-pass (max, then sum), top-p is a full
+ * sort.  No blocking, no online softmax, no fusion.  OpenMP only parallelises
+ * over independent (head, query block) units; it never changes the order of a
+ * floating-point reduction.
+ *
+ * Passage followed by each function is named in its comment:
+ *   "Eq. mean-pooled drift"  = the mean-pooled approximation of the query-key
+ *                              drift in the Temporal Mask Reuse section,
+ *   "Eq. full-token drift"   = the token-level drift it approximates,
+ *   "Algorithm 1"            = the Temporal Mask Reuse procedure (appendix),
+ *   "Observation I/II"       = the minimal cumulative-mass (top-p) set.
+ *
+ * Pinning status (tests/test_oracle_pins.py):
+ *   token mean, drift, decision, gate ........ pinned (closed forms, the paper's
+ *                                              cache-size example, Algorithm 1
+ *                                              state table)
+ *   block pooling, softmax, top-p ............ pinned (brute-force subset search,
+ *                                              uniform-row closed form, limits)
+ *   masked attention ......................... pinned (dense brute force, library
+ *                                              attention, closed forms)
+ *   fidelity of the block-importance estimator to the paper's third-party
+ *   backbones (antidiagonal scoring / k-means) ........ parity unpinned: the
+ *   paper does not define them; the estimator here is mean-pooled Q.K^T.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_FORCE_REFRESH 1u
+#define ORACLE_FORCE_DENSE 2u
+
+static double bf16_to_double(uint16_t h) {
+  uint32_t u = ((uint32_t)h) << 16;
+  float f;
+  memcpy(&f, &u, sizeof f);
+  return (double)f;
+}
+
+/* ---------------------------------------------------------------------------
+ * O1. Token mean (Algorithm 1, line 1; Eq. mean-pooled drift):
+ *     mean[r][d] = (1/N) * sum_{i<N} X[r][i][d].   X is bf16 [R][N][D].
+ * ------------------------------------------------------------------------ */
+void oracle_token_mean(const uint16_t *X, int R, int N, int D, double *mean) {
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int r = 0; r < R; ++r)
+    for (int d = 0; d < D; ++d) {
+      double s = 0.0;
+      for (int i = 0; i < N; ++i) s += bf16_to_double(X[((size_t)r * N + i) * D + d]);
+      mean[(size_t)r * D + d] = s / (double)N;
+    }
+}
+
+/* ---------------------------------------------------------------------------
+ * O2. Mean-pooled drift (Eq. mean-pooled drift; Algorithm 1, drift line):
+ *     drift[r] = ||aq[r]-mq[r]||_1 + ||ak[r]-mk[r]||_1     (plain sums over D)
+ * ------------------------------------------------------------------------ */
+void oracle_pooled_drift(const double *aq, const double *ak, const double *mq, const double *mk,
+                         int R, int D, double *drift) {
+  for (int r = 0; r < R; ++r) {
+    double dq = 0.0, dk = 0.0;
+    for (int d = 0; d < D; ++d) dq += fabs(aq[(size_t)r * D + d] - mq[(size_t)r * D + d]);
+    for (int d = 0; d < D; ++d) dk += fabs(ak[(size_t)r * D + d] - mk[(size_t)r * D + d]);
+    drift[r] = dq + dk;
+  }
+}
+
+/* ---------------------------------------------------------------------------
+ * Full-token drift (Eq. full-token drift), analysis quantity only:
+ *     d[r] = (1/N) sum_i ( ||qa_i - qb_i||_1 + ||ka_i - kb_i||_1 )
+ * ------------------------------------------------------------------------ */
+void oracle_full_token_drift(const uint16_t *Qa, const uint16_t *Ka, const uint16_t *Qb,
+                             const uint16_t *Kb, int R, int N, int D, double *drift) {
+  for (int r = 0; r < R; ++r) {
+    double s = 0.0;
+    for (int i = 0; i < N; ++i) {
+      size_t o = ((size_t)r * N + i) * D;
+      double t = 0.0;
+      for (int d = 0; d < D; ++d) t += fabs(bf16_to_double(Qa[o + d]) - bf16_to_double(Qb[o + d]));
+      for (int d = 0; d < D; ++d) t += fabs(bf16_to_double(Ka[o + d]) - bf16_to_double(Kb[o + d]));
+      s += t;
+    }
+    drift[r] = s / (double)N;
+  }
+}
+
+/* ---------------------------------------------------------------------------
+ * O3. Refresh-or-reuse decision and anchor update (Algorithm 1; the layer gate
+ * of the Temporal Mask Reuse section, constants in the HEART-configurations
+ * appendix).
+ *   head-wise:  refresh = no anchor  OR  drift > delta      (strict)
+ *   gate (per batch entry, over its H heads, f = #refresh / H):
+ *       f < gate_lo  -> every head that has an anchor reuses
+ *       f > gate_hi  -> every head refreshes
+ *       otherwise head-wise decisions stand.
+ *     Heads without an anchor always refresh (no mask exists to reuse).
+ *     gate_lo = 0, gate_hi = 1 can never fire (strict inequalities).
+ *   on refresh: anchor <- current means, has_anchor <- 1; on reuse untouched.
+ * drift[r] is +inf where no anchor exists.
+ * ------------------------------------------------------------------------ */
+void oracle_decide(const double *mq, const double *mk, const double *delta, int B, int H, int D,
+                   double gate_lo, double gate_hi, uint32_t flags, double *aq, double *ak,
+                   uint8_t *has_anchor, double *drift, uint8_t *refresh) {
+  int R = B * H;
+  for (int r = 0; r < R; ++r) {
+    if (!has_anchor[r]) {
+      drift[r] = INFINITY;
+      refresh[r] = 1;
+    } else {
+      oracle_pooled_drift(aq + (size_t)r * D, ak + (size_t)r * D, mq + (size_t)r * D,
+                          mk + (size_t)r * D, 1, D, drift + r);
+      refresh[r] = (drift[r] > delta[r]) ? 1 : 0;
+    }
+    if (flags & ORACLE_FORCE_REFRESH) refresh[r] = 1;
+  }
+  for (int b = 0; b < B; ++b) {
+    int cnt = 0;
+    for (int h = 0; h < H; ++h) cnt += refresh[b * H + h];
+    double f = (double)cnt / (double)H;
+    if (f < gate_lo) {
+      for (int h = 0; h < H; ++h)
+        if (has_anchor[b * H + h]) refresh[b * H + h] = 0;
+    } else if (f > gate_hi) {
+      for (int h = 0; h < H; ++h) refresh[b * H + h] = 1;
+    }
+  }
+  for (int r = 0; r < R; ++r)
+    if (refresh[r]) {
+      memcpy(aq + (size_t)r * D, mq + (size_t)r * D, sizeof(double) * D);
+      memcpy(ak + (size_t)r * D, mk + (size_t)r * D, sizeof(double) * D);
+      has_anchor[r] = 1;
+    }
+}
+
+/* ---------------------------------------------------------------------------
+ * O4. Block pooling: pooled[r][I][d] = mean over the REAL tokens of block I,
+ *     i in [I*b, min((I+1)*b, N)).  The last block divides by its own count.
+ * ------------------------------------------------------------------------ */
+void oracle_block_pool(const uint16_t *X, int R, int N, int D, int b, double *pooled) {
+  int nb = (N + b - 1) / b;
+#pragma omp parallel for collapse(2) schedule(static)
+  for (int r = 0; r < R; ++r)
+    for (int I = 0; I < nb; ++I) {
+      int i0 = I * b, i1 = (I + 1) * b < N ? (I + 1) * b : N;
+      for (int d = 0; d < D; ++d) {
+        double s = 0.0;
+        for (int i = i0; i < i1; ++i) s += bf16_to_double(X[((size_t)r * N + i) * D + d]);
+        pooled[((size_t)r * nb + I) * D + d] = s / (double)(i1 - i0);
+      }
+    }
+}
+
+/* ---------------------------------------------------------------------------
+ * O5. Block scores and row softmax for one query block:
+ *     S[J] = scale * <qp, Kp[J]>,  P[J] = exp(S[J]-max S) / sum_J exp(S[J]-max S)
+ * (scaled dot product as in the appendix's query-key interaction; plain softmax
+ * over all key blocks, no causal mask, no weighting by block length).
+ * ------------------------------------------------------------------------ */
+void oracle_block_probs(const double *qp, const double *Kp, int nb, int D, double scale, double *P) {
+  double mx = -INFINITY;
+  for (int J = 0; J < nb; ++J) {
+    double s = 0.0;
+    for (int d = 0; d < D; ++d) s += qp[d] * Kp[(size_t)J * D + d];
+    P[J] = s * scale;
+    if (P[J] > mx) mx = P[J];
+  }
+  double z = 0.0;
+  for (int J = 0; J < nb; ++J) {
+    P[J] = exp(P[J] - mx);
+    z += P[J];
+  }
+  for (int J = 0; J < nb; ++J) P[J] /= z;
+}
+
+typedef struct {
+  double p;
+  int j;
+} oracle_pj;
+
+static int cmp_desc_p_asc_j(const void *a, const void *b) {
+  const oracle_pj *x = (const oracle_pj *)a, *y = (const oracle_pj *)b;
+  if (x->p > y->p) return -1;
+  if (x->p < y->p) return 1;
+  return (x->j > y->j) - (x->j < y->j);
+}
+
+/* ---------------------------------------------------------------------------
+ * O6. Top-p selection (Observation I: the minimal set whose cumulative mass
+ * reaches the threshold; Observation II: rank by importance, retain until the
+ * accumulated importance reaches tau).
+ *   order by (P descending, index ascending); c_k = sum of the first k;
+ *   k* = min{k>=1 : c_k >= tau};  tau >= 1, or never reached -> k* = n.
+ * keep[j] = 1 for the first k* of that order.  Returns k*.  Optionally reports
+ * c_{k*} and c_{k*-1} for the near-boundary checks of the parity tests.
+ * ------------------------------------------------------------------------ */
+int oracle_top_p(const double *P, int n, double tau, uint8_t *keep, double *c_at, double *c_before) {
+  if (n <= 0) return 0;
+  oracle_pj *v = (oracle_pj *)malloc(sizeof(oracle_pj) * (size_t)n);
+  for (int j = 0; j < n; ++j) {
+    v[j].p = P[j];
+    v[j].j = j;
+  }
+  qsort(v, (size_t)n, sizeof(oracle_pj), cmp_desc_p_asc_j);
+  int kstar = n;
+  double c = 0.0, cprev = 0.0, c_hit = 0.0, c_hit_prev = 0.0;
+  int hit = 0;
+  for (int k = 1; k <= n; ++k) {
+    cprev = c;
+    c += v[k - 1].p;
+    if (!hit && !(tau >= 1.0) && c >= tau) {
+      kstar = k;
+      hit = 1;
+      c_hit = c;
+      c_hit_prev = cprev;
+    }
+  }
+  if (!hit) {
+    c_hit = c;
+    c_hit_prev = cprev;
+  }
+  memset(keep, 0, (size_t)n);
+  for (int k = 0; k < kstar; ++k) keep[v[k].j] = 1;
+  if (c_at) *c_at = c_hit;
+  if (c_before) *c_before = c_hit_prev;
+  free(v);
+  return kstar;
+}
+
+/* ---------------------------------------------------------------------------
+ * O4-O6 for the refreshed heads: writes, per (r, I), the canonical bit mask
+ * (bit J%32 of word J/32), the ascending index list and the count.  Heads with
+ * refresh[r] == 0 are left untouched (Algorithm 1, reuse branch).
+ * refresh == NULL means all heads.  ORACLE_FORCE_DENSE keeps every block.
+ * ------------------------------------------------------------------------ */
+void oracle_predict_mask(const uint16_t *Q, const uint16_t *K, int R, int N, int D, int b,
+                         double scale, const double *tau, const uint8_t *refresh, uint32_t flags,
+                         uint32_t *mask_bits, int32_t *kv_idx, int32_t *kv_cnt, int idx_stride) {
+  int nb = (N + b - 1) / b;
+  int W = (nb + 31) / 32;
+  if (!(scale > 0.0)) scale = 1.0 / sqrt((double)D);
+  for (int r = 0; r < R; ++r) {
+    if (refresh && !refresh[r]) continue;
+    double *Qp = (double *)malloc(sizeof(double) * (size_t)nb * D);
+    double *Kp = (double *)malloc(sizeof(double) * (size_t)nb * D);
+    oracle_block_pool(Q + (size_t)r * N * D, 1, N, D, b, Qp);
+    oracle_block_pool(K + (size_t)r * N * D, 1, N, D, b, Kp);
+#pragma omp parallel
+    {
+      double *P = (double *)malloc(sizeof(double) * (size_t)nb);
+      uint8_t *keep = (uint8_t *)malloc((size_t)nb);
+#pragma omp for schedule(static)
+      for (int I = 0; I < nb; ++I) {
+        oracle_block_probs(Qp + (size_t)I * D, Kp, nb, D, scale, P);
+        double t = (flags & ORACLE_FORCE_DENSE) ? 1.0 : tau[r];
+        oracle_top_p(P, nb, t, keep, NULL, NULL);
+        uint32_t *bits = mask_bits + ((size_t)r * nb + I) * W;
+        int32_t *idx = kv_idx + ((size_t)r * nb + I) * idx_stride;
+        memset(bits, 0, sizeof(uint32_t) * (size_t)W);
+        int c = 0;
+        for (int J = 0; J < nb; ++J)
+          if (keep[J]) {
+            bits[J >> 5] |= 1u << (J & 31);
+            idx[c++] = J;
+          }
+        kv_cnt[(size_t)r * nb + I] = c;
+      }
+      free(P);
+      free(keep);
+    }
+    free(Qp);
+    free(Kp);
+  }
+}
+
+/* One row of block probabilities for (r, I), for the parity checker. */
+void oracle_probs_row(const uint16_t *Q, const uint16_t *K, int N, int D, int b, double scale, int r,
+                      int I, double *P) {
+  int nb = (N + b - 1) / b;
+  if (!(scale > 0.0)) scale = 1.0 / sqrt((double)D);
+  double *Qp = (double *)malloc(sizeof(double) * (size_t)nb * D);
+  double *Kp = (double *)malloc(sizeof(double) * (size_t)nb * D);
+  oracle_block_pool(Q + (size_t)r * N * D, 1, N, D, b, Qp);
+  oracle_block_pool(K + (size_t)r * N * D, 1, N, D, b, Kp);
+  oracle_block_probs(Qp + (size_t)I * D, Kp, nb, D, scale, P);
+  free(Qp);
+  free(Kp);
+}
+
+/* ---------------------------------------------------------------------------
+ * O7. Masked attention for one (r, I) query block.  For each real query token
+ * i of block I:  logits l_j = scale*<q_i,k_j> over every real key j (j < N) of
+ * every listed key block;  o_i = sum_j softmax(l)_j v_j;  lse_i = max + log sum
+ * exp(l - max).  An empty list gives o_i = 0, lse_i = -inf.
+ * out is [b][D] (rows past N untouched), lse is [b].
+ * ------------------------------------------------------------------------ */
+void oracle_attn_block(const uint16_t *Q, const uint16_t *K, const uint16_t *V, int N, int D, int b,
+                       double scale, int r, int I, const int32_t *idx, int cnt, double *out,
+                       double *lse) {
+  if (!(scale > 0.0)) scale = 1.0 / sqrt((double)D);
+  size_t base = (size_t)r * N * D;
+  int i0 = I * b, i1 = (I + 1) * b < N ? (I + 1) * b : N;
+  int maxkeys = cnt * b;
+  double *l = (double *)malloc(sizeof(double) * (size_t)(maxkeys > 0 ? maxkeys : 1));
+  int *key = (int *)malloc(sizeof(int) * (size_t)(maxkeys > 0 ? maxkeys : 1));
+  for (int i = i0; i < i1; ++i) {
+    int nk = 0;
+    double mx = -INFINITY;
+    for (int t = 0; t < cnt; ++t) {
+      int J = idx[t];
+      int j1 = (J + 1) * b < N ? (J + 1) * b : N;
+      for (int j = J * b; j < j1; ++j) {
+        double s = 0.0;
+        for (int d = 0; d < D; ++d)
+          s += bf16_to_double(Q[base + (size_t)i * D + d]) * bf16_to_double(K[base + (size_t)j * D + d]);
+        l[nk] = s * scale;
+        key[nk] = j;
+        if (l[nk] > mx) mx = l[nk];
+        ++nk;
+      }
+    }
+    double *o = out + (size_t)(i - i0) * D;
+    for (int d = 0; d < D; ++d) o[d] = 0.0;
+    if (nk == 0) {
+      if (lse) lse[i - i0] = -INFINITY;
+      continue;
+    }
+    double z = 0.0;
+    for (int t = 0; t < nk; ++t) {
+      l[t] = exp(l[t] - mx);
+      z += l[t];
+    }
+    for (int t = 0; t < nk; ++t) {
+      double w = l[t] / z;
+      const uint16_t *v = V + base + (size_t)key[t] * D;
+      for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(v[d]);
+    }
+    if (lse) lse[i - i0] = mx + log(z);
+  }
+  free(l);
+  free(key);
+}
+
+/* O7 over a list of (r, I) query blocks; out is [n_rows][b][D], lse [n_rows][b].
+ * Rows past N in a ragged last block are left as they were. */
+void oracle_attn_rows(const uint16_t *Q, const uint16_t *K, const uint16_t *V, int N, int D, int b,
+                      double scale, const int32_t *kv_idx, const int32_t *kv_cnt, int idx_stride,
+                      const int32_t *rows_r, const int32_t *rows_I, int n_rows, double *out,
+                      double *lse) {
+  int nb = (N + b - 1) / b;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int t = 0; t < n_rows; ++t) {
+    int r = rows_r[t], I = rows_I[t];
+    size_t row = (size_t)r * nb + I;
+    oracle_attn_block(Q, K, V, N, D, b, scale, r, I, kv_idx + row * idx_stride, kv_cnt[row],
+                      out + (size_t)t * b * D, lse ? lse + (size_t)t * b : NULL);
+  }
+}
+
+/* O7 over every (r, I); O is fp64 [R][N][D], lse [R][N]. */
+void oracle_block_sparse_attn(const uint16_t *Q, const uint16_t *K, const uint16_t *V, int R, int N,
+                              int D, int b, double scale, const int32_t *kv_idx,
+                              const int32_t *kv_cnt, int idx_stride, double *O, double *lse) {
+  int nb = (N + b - 1) / b;
+#pragma omp parallel
+  {
+    double *tmp = (double *)malloc(sizeof(double) * (size_t)b * D);
+    double *tl = (double *)malloc(sizeof(double) * (size_t)b);
+#pragma omp for collapse(2) schedule(dynamic, 1)
+    for (int r = 0; r < R; ++r)
+      for (int I = 0; I < nb; ++I) {
+        size_t row = (size_t)r * nb + I;
+        oracle_attn_block(Q, K, V, N, D, b, scale, r, I, kv_idx + row * idx_stride, kv_cnt[row], tmp, tl);
+        int i0 = I * b, i1 = (I + 1) * b < N ? (I + 1) * b : N;
+        memcpy(O + ((size_t)r * N + i0) * D, tmp, sizeof(double) * (size_t)(i1 - i0) * D);
+        if (lse) memcpy(lse + (size_t)r * N + i0, tl, sizeof(double) * (size_t)(i1 - i0));
+      }
+    free(tmp);
+    free(tl);
+  }
+}
+
+/* Dense softmax attention by its textbook definition (no block structure at
+ * all), used by the tests as the brute-force pin of O7 with a full mask. */
+void oracle_dense_attn(const uint16_t *Q, const uint16_t *K, const uint16_t *V, int R, int N, int D,
+                       double scale, double *O) {
+  if (!(scale > 0.0)) scale = 1.0 / sqrt((double)D);
+#pragma omp parallel
+  {
+    double *l = (double *)malloc(sizeof(double) * (size_t)N);
+#pragma omp for collapse(2) schedule(static)
+    for (int r = 0; r < R; ++r)
+      for (int i = 0; i < N; ++i) {
+        size_t base = (size_t)r * N * D;
+        double mx = -INFINITY;
+        for (int j = 0; j < N; ++j) {
+          double s = 0.0;
+          for (int d = 0; d < D; ++d)
+            s += bf16_to_double(Q[base + (size_t)i * D + d]) * bf16_to_double(K[base + (size_t)j * D + d]);
+          l[j] = s * scale;
+          if (l[j] > mx) mx = l[j];
+        }
+        double z = 0.0;
+        for (int j = 0; j < N; ++j) z += exp(l[j] - mx);
+        double *o = O + base + (size_t)i * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        for (int j = 0; j < N; ++j) {
+          double w = exp(l[j] - mx) / z;
+          for (int d = 0; d < D; ++d) o[d] += w * bf16_to_double(V[base + (size_t)j * D + d]);
+        }
+      }
+    free(l);
+  }
+}
+
+/* ---------------------------------------------------------------------------
+ * O8. One layer-step = O1 -> O2 -> O3 -> (O4-O6 for refreshed heads) -> O7,
+ * with the TMR state (anchors, has_anchor, masks) carried by the caller.
+ * ORACLE_FORCE_DENSE: dense warm-up step -- attention over every block, TMR
+ * state untouched, refresh reported 0 and drift +inf.
+ * If O == NULL the attention is skipped (state and decisions only).
+ * ------------------------------------------------------------------------ */
+void oracle_step(const uint16_t *Q, const uint16_t *K, const uint16_t *V, int B, int H, int N, int D,
+                 int b, double scale, double gate_lo, double gate_hi, uint32_t flags,
+                 const double *delta, const double *tau, double *aq, double *ak, uint8_t *has_anchor,
+                 uint32_t *mask_bits, int32_t *kv_idx, int32_t *kv_cnt, int idx_stride, double *O,
+                 double *lse, double *drift, uint8_t *refresh) {
+  int R = B * H;
+  int nb = (N + b - 1) / b;
+  if (flags & ORACLE_FORCE_DENSE) {
+    for (int r = 0; r < R; ++r) {
+      drift[r] = INFINITY;
+      refresh[r] = 0;
+    }
+    if (O) {
+      int32_t *fi = (int32_t *)malloc(sizeof(int32_t) * (size_t)R * nb * nb);
+      int32_t *fc = (int32_t *)malloc(sizeof(int32_t) * (size_t)R * nb);
+      for (size_t row = 0; row < (size_t)R * nb; ++row) {
+        fc[row] = nb;
+        for (int J = 0; J < nb; ++J) fi[row * nb + J] = J;
+      }
+      oracle_block_sparse_attn(Q, K, V, R, N, D, b, scale, fi, fc, nb, O, lse);
+      free(fi);
+      free(fc);
+    }
+    return;
+  }
+  double *mq = (double *)malloc(sizeof(double) * (size_t)R * D);
+  double *mk = (double *)malloc(sizeof(double) * (size_t)R * D);
+  oracle_token_mean(Q, R, N, D, mq);
+  oracle_token_mean(K, R, N, D, mk);
+  oracle_decide(mq, mk, delta, B, H, D, gate_lo, gate_hi, flags, aq, ak, has_anchor, drift, refresh);
+  oracle_predict_mask(Q, K, R, N, D, b, scale, tau, refresh, 0u, mask_bits, kv_idx, kv_cnt, idx_stride);
+  if (O) oracle_block_sparse_attn(Q, K, V, R, N, D, b, scale, kv_idx, kv_cnt, idx_stride, O, lse);
+  free(mq);
+  free(mk);
+}

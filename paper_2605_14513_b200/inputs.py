@@ -1,0 +1,219 @@
+"""Seeded synthetic inputs for the HEART hot path (shared by tests, smoke, bench).
+
+This module holds NONE of the method's arithmetic: it only manufactures the
+bf16 Q/K/V tensors and the per-head parameter vectors (tau, delta, eps) that
+both the CUDA path and the CPU oracle are then given byte-for-byte.
+
+The tensors stand in for the query/key/value activations of the video
+diffusion transformers the paper measures on (the models and their weights are
+not needed for the hot path): same shapes (heads, latent grid, head_dim 128),
+locality-concentrated attention, slowly drifting across denoising steps.
+
+Recipe
+------
+* Noise is a counter-based generator (a 64-bit mixing hash of
+  (seed, tensor, step, flat element index) -> two 24-bit uniforms -> Box-Muller),
+  written with torch integer ops so the same code runs on CPU and CUDA and any
+  element can be regenerated independently of the rest.
+* Base tensors at step 0:  X = G + pos_scale * E_h(pos(i)),  G ~ N(0,1) iid,
+  pos(i) = (t, y, x) of token i in raster order (x fastest), E_h a 3-D
+  sinusoidal embedding (128 dims split 44/42/42 over t/y/x; sin/cos pairs with
+  geometric frequencies 10000^(-k/(d/2)) * (1 + 0.1 h)).  Q, K and V each get
+  their own G; all three share E_h, which makes q.k peak for nearby tokens.
+* Step t+1 = step t + eps_h * N(0,1) on an fp32 master copy; the tensors handed
+  out are the round-to-nearest-even bf16 of the master.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+import torch
+
+_M64 = (1 << 64) - 1
+_GOLDEN = 0x9E3779B97F4A7C15
+
+
+def _s64(x: int) -> int:
+    x &= _M64
+    return x - (1 << 64) if x >= (1 << 63) else x
+
+
+def _lsr(z: torch.Tensor, s: int) -> torch.Tensor:
+    return (z >> s) & ((1 << (64 - s)) - 1)
+
+
+def _mix(z: torch.Tensor) -> torch.Tensor:
+    z = (z ^ _lsr(z, 30)) * _s64(0xBF58476D1CE4E5B9)
+    z = (z ^ _lsr(z, 27)) * _s64(0x94D049BB133111EB)
+    return z ^ _lsr(z, 31)
+
+
+def _stream_key(seed: int, tensor_id: int, step: int) -> int:
+    k = (seed * 0xD1342543DE82EF95 + tensor_id * 0xAF251AF3B0F025B5 + step * 0x2545F4914F6CDD1D + 0x1234567) & _M64
+    # one scalar round of the same mixer, in Python integers
+    k = ((k ^ (k >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    k = ((k ^ (k >> 27)) * 0x94D049BB133111EB) & _M64
+    return k ^ (k >> 31)
+
+
+def normal(seed: int, tensor_id: int, step: int, start: int, count: int, device) -> torch.Tensor:
+    """`count` standard normals for flat element indices [start, start+count)."""
+    idx = torch.arange(start, start + count, dtype=torch.int64, device=device)
+    z = _mix((idx + 1) * _s64(_GOLDEN) + _s64(_stream_key(seed, tensor_id, step)))
+    u1 = (_lsr(z, 40).to(torch.float32) + 0.5) * (1.0 / (1 << 24))
+    u2 = ((z & 0xFFFFFF).to(torch.float32) + 0.5) * (1.0 / (1 << 24))
+    return torch.sqrt(-2.0 * torch.log(u1)) * torch.cos((2.0 * math.pi) * u2)
+
+
+def positional(grid, D: int, head: int, device) -> torch.Tensor:
+    """E_h(pos(i)) for every token of the raster-ordered grid -> [N, D] fp32."""
+    T, Y, X = grid
+    split = (44, 42, 42)
+    assert D == sum(split)
+    t = torch.arange(T, device=device, dtype=torch.float32).view(T, 1, 1).expand(T, Y, X).reshape(-1)
+    y = torch.arange(Y, device=device, dtype=torch.float32).view(1, Y, 1).expand(T, Y, X).reshape(-1)
+    x = torch.arange(X, device=device, dtype=torch.float32).view(1, 1, X).expand(T, Y, X).reshape(-1)
+    parts = []
+    for coord, d in zip((t, y, x), split):
+        half = d // 2
+        k = torch.arange(half, device=device, dtype=torch.float32)
+        w = torch.pow(torch.tensor(10000.0, device=device), -k / half) * (1.0 + 0.1 * head)
+        ang = coord[:, None] * w[None, :]
+        parts += [torch.sin(ang), torch.cos(ang)]
+    return torch.cat(parts, dim=1)
+
+
+@dataclass
+class Workload:
+    """One of the benchmark configurations (shapes + per-head parameters)."""
+
+    name: str
+    H: int
+    grid: tuple
+    block: int
+    tau: np.ndarray
+    delta: np.ndarray
+    eps: np.ndarray
+    pos_scale: np.ndarray
+    seed: int
+    steps: int
+    B: int = 1
+    D: int = 128
+    note: str = ""
+
+    @property
+    def N(self) -> int:
+        return self.grid[0] * self.grid[1] * self.grid[2]
+
+    @property
+    def R(self) -> int:
+        return self.B * self.H
+
+    @property
+    def n_blocks(self) -> int:
+        return (self.N + self.block - 1) // self.block
+
+
+def _rw_drift(eps, k, N, D=128):
+    """Expected pooled L1 drift of a k-step Gaussian random walk (2 tensors x D dims)."""
+    return 2.0 * D * eps * math.sqrt(2.0 * k / (math.pi * N))
+
+
+def workload(name: str) -> Workload:
+    """The five configurations, by name or by 1-based index ("1".."5")."""
+    alias = {"1": "tiny", "2": "wan1.3b-480p", "3": "wan14b-480p", "4": "wan14b-720p", "5": "hunyuan-720p"}
+    name = alias.get(str(name), name)
+    if name == "tiny":
+        H = 2
+        return Workload(name, H, (2, 32, 32), 64, np.array([0.9, 0.95]), np.array([0.25, 0.25]),
+                        np.array([0.01, 0.3]), np.full(H, 2.5), seed=0, steps=2,
+                        note="step 0: both heads refresh (no anchor); step 1: only head 1 refreshes")
+    if name == "wan1.3b-480p":
+        H, grid = 12, (21, 30, 52)
+        rs = np.random.RandomState(2)
+        tau = rs.uniform(0.85, 0.98, H)
+        eps = np.exp(rs.uniform(math.log(0.003), math.log(0.3), H))
+        N = grid[0] * grid[1] * grid[2]
+        delta = np.full(H, _rw_drift(0.03, 5, N))
+        return Workload(name, H, grid, 64, tau, delta, eps, np.full(H, 2.6), seed=2, steps=50,
+                        note="shared delta = 5-step drift of the geometric-mid eps")
+    if name == "wan14b-480p":
+        H, grid = 40, (21, 30, 52)
+        rs = np.random.RandomState(3)
+        tau = rs.uniform(0.85, 0.98, H)
+        eps = np.where(np.arange(H) < H // 2, 0.005, 0.2)
+        return Workload(name, H, grid, 64, tau, np.full(H, 0.05), eps, np.full(H, 2.6), seed=3, steps=50,
+                        note="heads 0-19 stable (reuse), heads 20-39 drift (refresh) in every launch")
+    if name == "wan14b-720p":
+        H, grid = 40, (21, 45, 80)
+        N = grid[0] * grid[1] * grid[2]
+        rs = np.random.RandomState(4)
+        tau = _TAU_WAN14B_720P.copy()
+        eps = np.exp(rs.uniform(math.log(0.01), math.log(0.1), H))
+        period = np.array([4, 5, 6])[np.arange(H) % 3]
+        delta = np.array([_rw_drift(e, k - 0.5, N) for e, k in zip(eps, period)])
+        return Workload(name, H, grid, 128, tau, delta, eps, np.full(H, 2.6), seed=4, steps=50,
+                        note="tau_h preset for a ~15% global block budget; refresh period 4/5/6 steps")
+    if name == "hunyuan-720p":
+        H, grid = 24, (33, 45, 80)
+        rs = np.random.RandomState(5)
+        tau = rs.uniform(0.80, 0.97, H)
+        return Workload(name, H, grid, 128, tau, np.zeros(H), np.full(H, 0.05), np.full(H, 2.6), seed=5,
+                        steps=50, note="delta = 0: every head refreshes at every step")
+    raise ValueError(f"unknown workload {name!r}")
+
+
+# Per-head thresholds of the 720P Wan-14B-shaped workload (placeholder for an
+# EBC-calibrated table): uniform here, tuned so the realised block density of
+# the synthetic tensors is ~15 %.
+_TAU_WAN14B_720P = np.full(40, 0.90)
+
+
+def small_workload(H=3, grid=(3, 10, 14), block=64, seed=7, steps=3, tau=None, eps=None, delta=None,
+                   pos_scale=2.5, B=1) -> Workload:
+    """A few-tile case with a ragged last block, for parity tests the oracle runs in seconds."""
+    R = B * H
+    rs = np.random.RandomState(seed)
+    tau = np.asarray(tau if tau is not None else rs.uniform(0.6, 0.97, R), dtype=np.float64)
+    eps = np.asarray(eps if eps is not None else np.exp(rs.uniform(math.log(0.003), math.log(0.3), R)))
+    N = grid[0] * grid[1] * grid[2]
+    delta = np.asarray(delta if delta is not None else np.full(R, _rw_drift(0.03, 1.5, N)))
+    return Workload("small", H, grid, block, tau, delta, eps, np.full(R, float(pos_scale)), seed, steps, B=B)
+
+
+class Sequence:
+    """Q/K/V of a workload across denoising steps (fp32 masters, bf16 views)."""
+
+    def __init__(self, wl: Workload, device="cpu"):
+        self.wl, self.device, self.t = wl, torch.device(device), 0
+        R, N, D = wl.R, wl.N, wl.D
+        self.master = [torch.empty((R, N, D), dtype=torch.float32, device=self.device) for _ in range(3)]
+        for r in range(R):
+            E = positional(wl.grid, D, r % wl.H, self.device) * float(wl.pos_scale[r])
+            for tid in range(3):
+                g = normal(wl.seed, tid, 0, r * N * D, N * D, self.device).view(N, D)
+                self.master[tid][r] = g + E
+            del E
+
+    def advance(self):
+        """Move every tensor one denoising step: X += eps_h * N(0,1)."""
+        wl = self.wl
+        self.t += 1
+        N, D = wl.N, wl.D
+        for r in range(wl.R):
+            for tid in range(3):
+                g = normal(wl.seed, tid, self.t, r * N * D, N * D, self.device).view(N, D)
+                self.master[tid][r].add_(g, alpha=float(wl.eps[r]))
+
+    def bf16(self):
+        """(Q, K, V) as bf16 [B, H, N, D] tensors (fresh copies)."""
+        wl = self.wl
+        return tuple(m.to(torch.bfloat16).view(wl.B, wl.H, wl.N, wl.D) for m in self.master)
+
+
+def bits(x: torch.Tensor) -> np.ndarray:
+    """Raw bf16 bits of a tensor as a numpy uint16 array [R, N, D] (for the oracle)."""
+    x = x.detach().to("cpu").contiguous()
+    return x.view(torch.int16).numpy().view(np.uint16).reshape(-1, x.shape[-2], x.shape[-1])
