@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the HEART layer-step (drift + mask prediction + block-sparse attention) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload wan1.3b-480p] [--impl reference]
+
+A "step" is one heart_step call = one whole pass of the hot path over one denoising step of
+synthetic Q/K/V (seeded, shaped like the paper's Wan2.1 / HunyuanVideo activations), with the TMR
+state carried from step to step so refresh and reuse mix as in a real sweep.  Prints ONE JSON line.
+
+The path does not shard (one layer's heads could be split across GPUs with no exchange, but the
+north star is a single-GPU kernel library): with --gpus N every rank runs an independent replica
+("replicas only"), and `value` is the time per layer-step of the whole job = max-over-ranks step
+time / N.
+
+--impl reference times the CPU oracle (oracle/) as it stands on the host cores, on a bounded
+sample of the same workload, and prints the same line with "impl": "reference".
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "ms per layer-step (drift+mask+attn)"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="wan1.3b-480p")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-sample-rows", type=int, default=8, help="query blocks the CPU oracle attends per step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled every 200 ms while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}",
+                                       "--format=csv,noheader,nounits", "-lms", "200"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.p.terminate()
+        self.p.wait()
+        self.f.flush()
+        rows = [l.strip().split(", ") for l in open(self.f.name) if l.strip()]
+        os.unlink(self.f.name)
+        sm, mx, reasons = [], [], set()
+        for r in rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if v.strip().lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def retained_flops(torch, st, wl):
+    """4 * (real query rows) * (real key rows) * D summed over the retained pairs (never padding)."""
+    nb, b, N = wl.n_blocks, wl.block, wl.N
+    last = N - (nb - 1) * b
+    cnt = st.kv_cnt.to(torch.float64)                                    # [R, nb]
+    has_last = ((st.mask_bits[:, :, (nb - 1) // 32] >> ((nb - 1) % 32)) & 1).to(torch.float64)
+    keys = cnt * b - has_last * (b - last)                               # real key rows per query block
+    qrows = torch.full((nb,), float(b), dtype=torch.float64, device=cnt.device)
+    qrows[nb - 1] = last
+    return float(4.0 * wl.D * (keys * qrows[None, :]).sum().item()), float(cnt.sum().item())
+
+
+def run_ours(args, rank, world):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_14513_b200 import heart, inputs
+
+    heart.lib()  # fails loudly if the CUDA library is missing
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    pk = peaks()
+    wl = inputs.workload(args.workload)
+    K, W = args.steps, args.warmup
+    n_inputs = K + W
+
+    # ---- synthetic inputs, all resident in HBM before anything is timed
+    seq = inputs.Sequence(wl, dev)
+    steps_in = []
+    for t in range(n_inputs):
+        steps_in.append(seq.bf16())
+        if t + 1 < n_inputs:
+            seq.advance()
+    del seq
+    cfg = heart.make_config(wl.B, wl.H, wl.N, wl.block)
+    st, ws = heart.State(cfg, dev), heart.new_workspace(cfg, dev)
+    delta = torch.tensor(wl.delta, dtype=torch.float64, device=dev)
+    tau = torch.tensor(wl.tau, dtype=torch.float64, device=dev)
+    O = torch.empty_like(steps_in[0][0])
+    drift = torch.empty(wl.R, dtype=torch.float64, device=dev)
+    refresh = torch.empty(wl.R, dtype=torch.uint8, device=dev)
+
+    def step(t):
+        Q, Kt, V = steps_in[t]
+        heart.heart_step(cfg, Q, Kt, V, delta, tau, st, O, ws, drift_out=drift, refresh_out=refresh)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(W):
+        step(t)
+    torch.cuda.synchronize()
+    ckpt = st.state_dict()  # state after warm-up: the e2e and per-stage passes restart from here
+
+    # ---- timed region: exactly K steps, device-resident inputs, one event pair per step
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", "")
+    sampler = ClockSampler(uuid) if rank == 0 else None
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    launches = 0
+    barrier()
+    t_wall = time.perf_counter()
+    for k in range(K):
+        ev[k][0].record()
+        step(W + k)
+        ev[k][1].record()
+        launches += heart.heart_last_launch_count()
+    barrier()
+    wall_ms = (time.perf_counter() - t_wall) * 1e3
+    clocks = sampler.stop() if sampler else None
+    total_ms = ev[0][0].elapsed_time(ev[-1][1])
+    assert heart.heart_get_status(ws) == 0
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / K
+
+    # ---- per-stage pass: the same K steps as three C-ABI calls, one event pair per call
+    st.load_state_dict(ckpt)
+    stage_ev = []
+    flops_total = pairs_total = refreshed = 0.0
+    r2 = torch.empty_like(refresh)
+    for k in range(K):
+        Q, Kt, V = steps_in[W + k]
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        e[0].record()
+        heart.heart_drift(cfg, Q, Kt, delta, st, ws, refresh_out=r2)
+        e[1].record()
+        heart.heart_predict_mask(cfg, Q, Kt, tau, st, ws, refresh=r2)
+        e[2].record()
+        heart.heart_block_sparse_attn(cfg, Q, Kt, V, st.kv_idx, st.kv_cnt, O, ws)
+        e[3].record()
+        stage_ev.append(e)
+        torch.cuda.synchronize()
+        f, p = retained_flops(torch, st, wl)
+        flops_total += f
+        pairs_total += p
+        refreshed += float(r2.sum().item())
+    ms_drift = sum(e[0].elapsed_time(e[1]) for e in stage_ev) / K
+    ms_mask = sum(e[1].elapsed_time(e[2]) for e in stage_ev) / K
+    ms_attn = sum(e[2].elapsed_time(e[3]) for e in stage_ev) / K
+    flops_step = flops_total / K
+    density = pairs_total / K / (wl.R * wl.n_blocks ** 2)
+    dense_flops = 4.0 * wl.R * float(wl.N) ** 2 * wl.D
+    attn_tflops = flops_step / (ms_attn * 1e-3) / 1e12
+    stats_bytes = 4.0 * wl.R * wl.N * wl.D  # Q and K read once (bf16)
+
+    # ---- end-to-end pass: host (pinned) Q/K/V in, O/drift/refresh out, through heart_step_host
+    e2e = None
+    if not args.no_e2e:
+        Ke = min(K, max(1, int(6e9 // (4 * 2 * wl.R * wl.N * wl.D))))  # cap pinned memory at ~6 GB
+        host_in = [tuple(x.cpu().pin_memory() for x in steps_in[W + k]) for k in range(Ke)]
+        Oh = torch.empty(O.shape, dtype=O.dtype).pin_memory()
+        dh = torch.empty(wl.R, dtype=torch.float64).pin_memory()
+        rh = torch.empty(wl.R, dtype=torch.uint8).pin_memory()
+        staging = tuple(torch.empty_like(O) for _ in range(4))
+        st.load_state_dict(ckpt)
+        heart.heart_step_host(cfg, *host_in[0], delta, tau, st, Oh, staging, ws, drift_host=dh, refresh_host=rh)
+        st.load_state_dict(ckpt)
+        barrier()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for k in range(Ke):
+            heart.heart_step_host(cfg, *host_in[k], delta, tau, st, Oh, staging, ws, drift_host=dh, refresh_host=rh)
+        b_.record()
+        barrier()
+        e2e_ms = a.elapsed_time(b_) / Ke
+        if world > 1:
+            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tt.item())
+        tensor_bytes = 2 * wl.R * wl.N * wl.D
+        e2e = {"value": e2e_ms / world, "unit": "ms", "steps": Ke, "h2d_bytes_per_step": 3 * tensor_bytes,
+               "d2h_bytes_per_step": tensor_bytes + 9 * wl.R,
+               "api": "heart_step_host (pinned host Q/K/V in, O + drift + refresh out)"}
+        del host_in, staging
+
+    out = None
+    if rank == 0:
+        peak_tf = pk["bf16_tflops_sustained"]
+        roofline = {"kernel": "block-sparse attention", "bound": "tensor", "achieved": attn_tflops, "peak": peak_tf,
+                    "unit": "TFLOP/s", "frac": attn_tflops / peak_tf, "traffic": None,
+                    "peak_source": pk["source"] + " (sustained bf16 cuBLAS, kernel timed inside a long step)",
+                    "flops_per_launch": flops_step, "ms_per_launch": ms_attn}
+        hbm = stats_bytes / (ms_drift * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": ms_per_step / world, "unit": "ms", "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "grid": list(wl.grid), "D": wl.D,
+                       "block": wl.block, "n_blocks": wl.n_blocks, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                       "l2": "inputs larger than L2 (every step reads new Q/K/V tensors, >= 3x the 126 MB L2)"
+                       if 6 * wl.R * wl.N * wl.D > 126e6 else "L2-resident (tiny case): not a roofline number"},
+            "stages_ms": {"drift": ms_drift, "mask": ms_mask, "attention": ms_attn,
+                          "sum_of_separate_calls": ms_drift + ms_mask + ms_attn},
+            "density": density, "refresh_rate": refreshed / (K * wl.R),
+            "retained_tflops": attn_tflops, "retained_tflops_vs_bf16_peak": attn_tflops / pk["bf16_tflops"],
+            "dense_equivalent_tflops": dense_flops / (ms_attn * 1e-3) / 1e12,
+            "dense_equivalent_speedup_at_same_throughput": dense_flops / flops_step,
+            "roofline": roofline,
+            "roofline_stats": {"kernel": "block sums + drift (heart_drift)", "bound": "hbm", "achieved": hbm,
+                               "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm / pk["hbm_gbs"],
+                               "frac_of_nominal_8TBps": hbm / 8000.0, "bytes_per_launch": stats_bytes,
+                               "ms_per_launch": ms_drift},
+            "gpu_launches": launches, "wall_ms_timed_region": wall_ms, "clocks": clocks, "e2e": e2e,
+        }
+    return out, (wl, steps_in, W)
+
+
+def oracle_sample_step(oracle, inputs, np, wl, ost, Qb, Kb, Vb, rs, n_rows):
+    """One oracle layer-step on a bounded sample: drift + decision + masks in full, attention on
+    n_rows query blocks, its time scaled by retained pairs.  Returns (seconds extrapolated, seconds spent)."""
+    t0 = time.perf_counter()
+    oracle.step(Qb, Kb, Vb, wl.delta, wl.tau, ost, want_O=False)
+    t1 = time.perf_counter()
+    rr = rs.randint(0, wl.R, n_rows).astype(np.int32)
+    II = rs.randint(0, wl.n_blocks, n_rows).astype(np.int32)
+    oracle.attn_rows(Qb, Kb, Vb, wl.block, ost.kv_idx, ost.kv_cnt, rr, II)
+    t2 = time.perf_counter()
+    sampled = float(ost.kv_cnt[rr, II].sum())
+    scale = float(ost.kv_cnt.sum()) / max(sampled, 1.0)
+    return (t1 - t0) + (t2 - t1) * scale, t2 - t0
+
+
+def run_reference(args):
+    """The oracle as it stands, on the host cores (rank 0 only)."""
+    import numpy as np
+
+    from oracle import heart_oracle as oracle
+    from paper_2605_14513_b200 import inputs
+
+    oracle.build()
+    wl = inputs.workload(args.workload)
+    K, W = args.steps, args.warmup
+    seq = inputs.Sequence(wl, "cpu")
+    ost = oracle.State(wl.B, wl.H, wl.N, wl.D, wl.block)
+    rs = np.random.RandomState(0)
+    est, spent = [], 0.0
+    for t in range(W + K):
+        Qb, Kb, Vb = (inputs.bits(x) for x in seq.bf16())
+        e, s = oracle_sample_step(oracle, inputs, np, wl, ost, Qb, Kb, Vb, rs, args.cpu_sample_rows)
+        if t >= W:
+            est.append(e)
+            spent += s
+        if t + 1 < W + K:
+            seq.advance()
+    ms = 1e3 * sum(est) / K
+    cores = os.cpu_count()
+    sample = (f"per step: token means, decision and masks in full; attention on {args.cpu_sample_rows} random "
+              f"query blocks scaled by retained pairs ({spent:.1f} s of CPU work in {K} steps)")
+    return {"impl": "reference", "metric": METRIC, "value": ms, "unit": "ms", "n_gpus": args.gpus, "steps": K,
+            "warmup": W, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "grid": list(wl.grid), "D": wl.D,
+                       "block": wl.block, "n_blocks": wl.n_blocks},
+            "cpu_baseline": {"value": ms, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": ms, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def cpu_baseline(args, wl, steps_in, W):
+    """The oracle timed on the host cores on a bounded sample of the benchmark's own inputs."""
+    import numpy as np
+
+    from oracle import heart_oracle as oracle
+    from paper_2605_14513_b200 import inputs
+
+    oracle.build()
+    ost = oracle.State(wl.B, wl.H, wl.N, wl.D, wl.block)
+    rs = np.random.RandomState(0)
+    est, spent, n = [], 0.0, 0
+    budget = 25.0
+    # step 0 builds the anchors and masks (all heads refresh); later steps show the steady mix
+    for t in range(min(len(steps_in), W + 3)):
+        Qb, Kb, Vb = (inputs.bits(x) for x in steps_in[t])
+        e, s = oracle_sample_step(oracle, inputs, np, wl, ost, Qb, Kb, Vb, rs, args.cpu_sample_rows)
+        spent += s
+        if t >= 1:
+            est.append(e)
+        n += 1
+        if spent > budget:
+            break
+    if not est:
+        est = [e]
+    ms = 1e3 * sum(est) / len(est)
+    return {"value": ms, "unit": "ms", "cores": os.cpu_count(), "kind": "oracle",
+            "sample": (f"{n} steps of the same inputs ({len(est)} after the all-refresh first step averaged); per step: "
+                       f"token means, decision and masks in full, attention on {args.cpu_sample_rows} random query blocks "
+                       f"scaled by retained pairs; {spent:.1f} s of CPU work")}
+
+
+def main():
+    args = parse()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+    out, (wl, steps_in, W) = run_ours(args, rank, world)
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_baseline(args, wl, steps_in, W)
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,158 @@
+/*
+ * heart.h -- C ABI of the B200 (sm_100a) HEART sparse-attention hot path.
+ *
+ * One layer-step of head-wise adaptive block-sparse attention for video
+ * diffusion transformers:
+ *   (a) Temporal Mask Reuse: mean-pooled query/key drift of every head against
+ *       its cached anchor step and the refresh-or-reuse decision
+ *       (Temporal Mask Reuse section, Eq. mean-pooled drift; Algorithm 1);
+ *   (b) block-importance mask prediction for the refreshed heads: block-pooled
+ *       Q.K^T scores, row softmax, cumulative top-p selection with each head's
+ *       own threshold tau_h (Observation II; the minimal cumulative-mass set of
+ *       Observation I; tau_h is the output of the offline calibration, an input
+ *       here);
+ *   (c) block-sparse attention over the retained (query block, key block) pairs
+ *       with online softmax.
+ *
+ * Conventions
+ *   - Every pointer below is a DEVICE pointer owned by the caller unless it is
+ *     marked "host".  The library never allocates or frees device memory and
+ *     keeps no state between calls; all state lives in heart_state.
+ *   - Every call except heart_get_status is asynchronous on `stream` and never
+ *     synchronises.  Arguments are validated on the host before any launch;
+ *     on a host-detected error nothing is launched and no state changes.
+ *   - R = B*H "head rows"; n_b = ceil(N / block); W = ceil(n_b / 32).
+ *   - Q, K, V, O are bf16 with head_dim contiguous; the element strides of the
+ *     other three dimensions are given in heart_config (0,0,0 selects the
+ *     contiguous [B,H,N,D] layout).  Base pointers must be 16-byte aligned and
+ *     strides multiples of 8 elements.
+ *   - Return value: HEART_OK or one of the HEART_ERR_* codes (never throws,
+ *     never traps, never exits).
+ */
+#ifndef HEART_H_
+#define HEART_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef void *heart_stream_t; /* a cudaStream_t (NULL = the legacy default stream) */
+
+enum {
+  HEART_OK = 0,
+  HEART_ERR_INVALID = 1,      /* null pointer, bad size/stride/alignment               */
+  HEART_ERR_UNSUPPORTED = 2,  /* D != 128, block not in {64,128}, n_b > 1024            */
+  HEART_ERR_CUDA = 3,         /* a CUDA call or launch failed (see heart_strerror)      */
+  HEART_ERR_DEVICE_CHECK = 4  /* a device-side check failed: bad index-list entry or a  */
+                              /* bounded wait ran out; only via heart_get_status        */
+};
+
+#define HEART_FORCE_REFRESH 1u /* every head refreshes this step (decision overridden)  */
+#define HEART_FORCE_DENSE 2u   /* dense warm-up step (the baselines' first denoising    */
+                               /* steps): attention over all blocks, TMR state untouched */
+
+#define HEART_MAX_BLOCKS 1024  /* largest supported n_b */
+
+typedef struct {
+  int32_t B, H, N, D;      /* D must be 128                                                */
+  int32_t block;           /* 64 or 128 tokens; query and key blocks are equal             */
+  int64_t stride_b, stride_h, stride_n; /* elements; all 0 = contiguous [B,H,N,D]          */
+  double scale;            /* logit scale; <= 0 selects 1/sqrt(D) (query-key interaction   */
+                           /* of the appendix)                                             */
+  double gate_lo, gate_hi; /* layer gate on the refreshed-head fraction (0.4 / 0.8 in the  */
+                           /* appendix); lo = 0, hi = 1 disables it                        */
+  int32_t idx_stride;      /* row pitch of kv_idx in entries, >= n_b                       */
+  uint32_t flags;          /* HEART_FORCE_*                                                */
+} heart_config;
+
+/* TMR state of one layer (Algorithm 1: cached anchor features and anchor mask). */
+typedef struct {
+  double *anchor_q, *anchor_k; /* [R, D]  token-mean Q and K at each head's anchor step    */
+  uint8_t *has_anchor;         /* [R]     0 = "no cached anchor exists"                    */
+  uint32_t *mask_bits;         /* [R, n_b, W] bit J%32 of word J/32 = pair (I,J) retained  */
+  int32_t *kv_idx;             /* [R, n_b, idx_stride] retained key blocks, ascending      */
+  int32_t *kv_cnt;             /* [R, n_b] number of retained key blocks per query block   */
+} heart_state;
+
+/* Bytes of scratch every compute call needs (block sums, means, flags, status
+ * word).  Host-only; returns 0 for an invalid or unsupported config.  The caller
+ * allocates it once (256-byte aligned) and zero-fills it before first use. */
+size_t heart_workspace_bytes(const heart_config *cfg /* host */);
+
+/* Clears has_anchor (and zeroes kv_cnt) so the next step refreshes every head
+ * (Algorithm 1, "no cached anchor exists"). */
+int heart_state_reset(const heart_config *cfg, heart_state *st /* host struct */, heart_stream_t stream);
+
+/* (a) Temporal Mask Reuse decision -- Eq. mean-pooled drift, Algorithm 1, layer gate.
+ *   mean_q[r,:] = (1/N) sum_i Q[r,i,:]  (same for K), fp64;
+ *   drift[r]    = ||anchor_q[r]-mean_q[r]||_1 + ||anchor_k[r]-mean_k[r]||_1   (+inf if no anchor);
+ *   refresh[r]  = !has_anchor[r] || drift[r] > delta[r]   (strict; then the gate per batch entry:
+ *                 fraction < gate_lo -> anchored heads reuse, fraction > gate_hi -> all refresh);
+ *   refreshed heads: anchor <- current means, has_anchor <- 1.
+ * delta [R] fp64 (a negative entry always refreshes).  drift_out [R] fp64 and refresh_out [R] u8
+ * may each be NULL.  Also leaves the per-block sums of Q and K in the workspace. */
+int heart_drift(const heart_config *cfg, const void *Q, const void *K, const double *delta,
+                heart_state *st, double *drift_out, uint8_t *refresh_out, void *workspace,
+                heart_stream_t stream);
+
+/* (b) Mask prediction for the heads with refresh[r] != 0 (NULL = all heads) -- Observation II.
+ *   Qp[r,I,:] = mean of the real tokens of block I (same for Kp), fp64;
+ *   P[r,I,:]  = softmax_J( scale * <Qp[r,I], Kp[r,J]> );
+ *   keep the first k* blocks in (P descending, J ascending) order, k* = min{k>=1: cum mass >= tau[r]};
+ *   tau[r] >= 1 (or a mass that never reaches tau) keeps all n_b blocks; at least one is kept.
+ * Writes mask_bits, kv_idx (ascending), kv_cnt of those heads; other heads are untouched.
+ * tau [R] fp64. */
+int heart_predict_mask(const heart_config *cfg, const void *Q, const void *K, const double *tau,
+                       const uint8_t *refresh, heart_state *st, void *workspace,
+                       heart_stream_t stream);
+
+/* (c) Block-sparse attention with online softmax over the listed pairs.
+ *   For query token i of block I:  o_i = sum_j softmax_j(scale * <q_i,k_j>) v_j over the real keys
+ *   (j < N) of the key blocks kv_idx[r,I,0..kv_cnt[r,I]).  bf16 in, fp32 accumulate, bf16 out (RNE).
+ *   An empty list gives zeros (lse = -inf).  Rows i >= N are never written.
+ *   lse [R, N] fp32 natural-log sum-exp of the scaled logits, or NULL.
+ *   Lists must hold distinct block indices in [0, n_b); entries out of range are skipped and
+ *   reported as HEART_ERR_DEVICE_CHECK through heart_get_status. */
+int heart_block_sparse_attn(const heart_config *cfg, const void *Q, const void *K, const void *V,
+                            const int32_t *kv_idx, const int32_t *kv_cnt, void *O, float *lse,
+                            void *workspace, heart_stream_t stream);
+
+/* One whole layer-step: heart_drift, then heart_predict_mask for the refreshed heads, then
+ * heart_block_sparse_attn with the (cached or new) lists -- all on `stream`, no host round trip
+ * (Algorithm 1 followed by the sparse attention it feeds).  Results equal the three calls made
+ * one after the other.  With HEART_FORCE_DENSE only dense attention runs (state untouched,
+ * refresh_out = 0, drift_out = +inf). */
+int heart_step(const heart_config *cfg, const void *Q, const void *K, const void *V,
+               const double *delta, const double *tau, heart_state *st, void *O, float *lse,
+               double *drift_out, uint8_t *refresh_out, void *workspace, heart_stream_t stream);
+
+/* heart_step for callers whose tensors live in HOST memory (the end-to-end path).
+ *   Q_host, K_host, V_host: bf16, contiguous [B,H,N,D] (cfg strides must be 0,0,0), ideally pinned;
+ *   O_host: bf16 [B,H,N,D] result; drift_host [R] fp64 and refresh_host [R] u8 may be NULL.
+ *   Q_dev, K_dev, V_dev, O_dev: caller-owned DEVICE staging buffers of B*H*N*D bf16 each.
+ * Enqueues on `stream`: three host-to-device copies, the step, the device-to-host copies of O,
+ * drift and refresh.  Does not synchronise: the host results are valid once `stream` has drained.
+ * delta, tau, st, workspace are device-side exactly as in heart_step. */
+int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_host, const void *V_host,
+                    const double *delta, const double *tau, heart_state *st, void *O_host,
+                    double *drift_host, uint8_t *refresh_host, void *Q_dev, void *K_dev, void *V_dev,
+                    void *O_dev, void *workspace, heart_stream_t stream);
+
+/* Synchronises `stream`, reads the workspace status word into *code_out (host) and clears it.
+ * The only call that blocks. */
+int heart_get_status(void *workspace, heart_stream_t stream, int32_t *code_out /* host */);
+
+/* Static description of a return code; for HEART_ERR_CUDA includes the last CUDA error text
+ * seen by the calling thread. */
+const char *heart_strerror(int code);
+
+/* Number of kernels the last compute call on this thread launched (for accounting). */
+int heart_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HEART_H_ */

@@ -1,0 +1,68 @@
+// Shared host/device helpers of the HEART CUDA library (geometry, workspace layout, status word).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "heart.h"
+
+namespace heart {
+
+constexpr int kD = 128;  // head_dim (fixed)
+
+// Geometry derived from a validated heart_config.
+struct Geom {
+  int B, H, R, N, block, nb, W, idx_stride;
+  long long sb, sh, sn;  // element strides of Q/K/V/O
+  double scale, gate_lo, gate_hi;
+  unsigned flags;
+};
+
+// Workspace layout (all offsets 256-byte aligned).
+struct Workspace {
+  int32_t *status;    // [64]   word 0: sticky device-check code; word 1: detail
+  double *bsum;       // [2][R][nb][D]  per-block sums of Q (0) and K (1)
+  double *mean;       // [2][R][D]      token means of the current step
+  double *part;       // [2][R]         L1 parts of the drift
+  uint8_t *pre;       // [R]            head-wise decision before the gate
+  uint8_t *refresh;   // [R]            final decision of the current step
+  double *drift;      // [R]
+  size_t bytes;
+};
+
+__host__ inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+__host__ inline Workspace carve(const Geom &g, void *base) {
+  Workspace w;
+  char *p = static_cast<char *>(base);
+  size_t off = 0;
+  w.status = reinterpret_cast<int32_t *>(p + off);
+  off += align256(64 * sizeof(int32_t));
+  w.bsum = reinterpret_cast<double *>(p + off);
+  off += align256(sizeof(double) * 2 * (size_t)g.R * g.nb * kD);
+  w.mean = reinterpret_cast<double *>(p + off);
+  off += align256(sizeof(double) * 2 * (size_t)g.R * kD);
+  w.part = reinterpret_cast<double *>(p + off);
+  off += align256(sizeof(double) * 2 * (size_t)g.R);
+  w.pre = reinterpret_cast<uint8_t *>(p + off);
+  off += align256((size_t)g.R);
+  w.refresh = reinterpret_cast<uint8_t *>(p + off);
+  off += align256((size_t)g.R);
+  w.drift = reinterpret_cast<double *>(p + off);
+  off += align256(sizeof(double) * (size_t)g.R);
+  w.bytes = off;
+  return w;
+}
+
+// Launchers (defined in the kernel files). Each returns the cudaError_t of its launches and
+// adds the number of kernels it launched to *launches.
+cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, double *bsum,
+                              cudaStream_t s, int *launches);
+cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta, heart_state st,
+                          double *drift_out, uint8_t *refresh_out, cudaStream_t s, int *launches);
+cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
+                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches);
+cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const void *V,
+                             const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,
+                             float *lse, int32_t *status, cudaStream_t s, int *launches);
+
+}  // namespace heart

@@ -1,0 +1,243 @@
+// C ABI of the HEART hot path: argument validation, workspace carving and kernel sequencing.
+// No device memory is allocated here and nothing synchronises except heart_get_status.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace heart;
+
+namespace {
+
+thread_local char g_errbuf[256] = "";
+thread_local int g_launches = 0;
+
+int cuda_fail(cudaError_t e, const char *where) {
+  snprintf(g_errbuf, sizeof g_errbuf, "CUDA error in %s: %s", where, cudaGetErrorString(e));
+  return HEART_ERR_CUDA;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates the shape part of a config and derives the geometry. Returns HEART_OK or an error.
+int make_geom(const heart_config *c, Geom *g) {
+  if (c == nullptr) return HEART_ERR_INVALID;
+  if (c->B <= 0 || c->H <= 0 || c->N <= 0) return HEART_ERR_INVALID;
+  if (c->D != kD) return HEART_ERR_UNSUPPORTED;
+  if (c->block != 64 && c->block != 128) return HEART_ERR_UNSUPPORTED;
+  g->B = c->B;
+  g->H = c->H;
+  g->R = c->B * c->H;
+  g->N = c->N;
+  g->block = c->block;
+  g->nb = (c->N + c->block - 1) / c->block;
+  if (g->nb > HEART_MAX_BLOCKS) return HEART_ERR_UNSUPPORTED;
+  g->W = (g->nb + 31) / 32;
+  if (c->stride_b == 0 && c->stride_h == 0 && c->stride_n == 0) {
+    g->sn = kD;
+    g->sh = (long long)c->N * kD;
+    g->sb = g->sh * c->H;
+  } else {
+    g->sb = c->stride_b;
+    g->sh = c->stride_h;
+    g->sn = c->stride_n;
+    if (g->sn < kD || g->sh <= 0 || g->sb <= 0) return HEART_ERR_INVALID;
+    if ((g->sn % 8) || (g->sh % 8) || (g->sb % 8)) return HEART_ERR_INVALID;
+  }
+  g->idx_stride = c->idx_stride;
+  if (g->idx_stride < g->nb) return HEART_ERR_INVALID;
+  g->scale = (c->scale > 0.0) ? c->scale : 1.0 / sqrt((double)kD);
+  g->gate_lo = c->gate_lo;
+  g->gate_hi = c->gate_hi;
+  if (isnan(g->gate_lo) || isnan(g->gate_hi)) return HEART_ERR_INVALID;
+  g->flags = c->flags;
+  return HEART_OK;
+}
+
+bool state_ok(const heart_state *st) {
+  return st && st->anchor_q && st->anchor_k && st->has_anchor && st->mask_bits && st->kv_idx && st->kv_cnt;
+}
+
+__global__ void fill_dense_outputs_kernel(int R, double *drift_out, uint8_t *refresh_out, uint8_t *refresh_ws) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r < R) {
+    if (drift_out) drift_out[r] = __longlong_as_double(0x7ff0000000000000LL);
+    if (refresh_out) refresh_out[r] = 0;
+    refresh_ws[r] = 0;
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t heart_workspace_bytes(const heart_config *cfg) {
+  Geom g;
+  if (make_geom(cfg, &g) != HEART_OK) return 0;
+  return carve(g, nullptr).bytes;
+}
+
+int heart_state_reset(const heart_config *cfg, heart_state *st, heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  if (!state_ok(st)) return HEART_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemsetAsync(st->has_anchor, 0, (size_t)g.R, s);
+  if (e != cudaSuccess) return cuda_fail(e, "heart_state_reset");
+  e = cudaMemsetAsync(st->kv_cnt, 0, sizeof(int32_t) * (size_t)g.R * g.nb, s);
+  if (e != cudaSuccess) return cuda_fail(e, "heart_state_reset");
+  return HEART_OK;
+}
+
+int heart_drift(const heart_config *cfg, const void *Q, const void *K, const double *delta,
+                heart_state *st, double *drift_out, uint8_t *refresh_out, void *workspace,
+                heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  if (!Q || !K || !delta || !workspace || !state_ok(st)) return HEART_ERR_INVALID;
+  if (!aligned16(Q) || !aligned16(K) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HEART_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  Workspace w = carve(g, workspace);
+  g_launches = 0;
+  cudaError_t e = launch_block_sums(g, Q, K, w.bsum, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "block_sums");
+  e = launch_decide(g, w, delta, *st, drift_out, refresh_out, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "decide");
+  return HEART_OK;
+}
+
+int heart_predict_mask(const heart_config *cfg, const void *Q, const void *K, const double *tau,
+                       const uint8_t *refresh, heart_state *st, void *workspace, heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  if (!Q || !K || !tau || !workspace || !state_ok(st)) return HEART_ERR_INVALID;
+  if (!aligned16(Q) || !aligned16(K) || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return HEART_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  Workspace w = carve(g, workspace);
+  g_launches = 0;
+  cudaError_t e = launch_block_sums(g, Q, K, w.bsum, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "block_sums");
+  e = launch_predict_mask(g, w, tau, refresh, *st, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
+  return HEART_OK;
+}
+
+int heart_block_sparse_attn(const heart_config *cfg, const void *Q, const void *K, const void *V,
+                            const int32_t *kv_idx, const int32_t *kv_cnt, void *O, float *lse,
+                            void *workspace, heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  const bool dense = (g.flags & HEART_FORCE_DENSE) != 0;
+  if (!Q || !K || !V || !O || !workspace) return HEART_ERR_INVALID;
+  if (!dense && (!kv_idx || !kv_cnt)) return HEART_ERR_INVALID;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return HEART_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  Workspace w = carve(g, workspace);
+  g_launches = 0;
+  cudaError_t e = launch_attention(g, Q, K, V, kv_idx, kv_cnt, dense, O, lse, w.status, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "attention");
+  return HEART_OK;
+}
+
+int heart_step(const heart_config *cfg, const void *Q, const void *K, const void *V,
+               const double *delta, const double *tau, heart_state *st, void *O, float *lse,
+               double *drift_out, uint8_t *refresh_out, void *workspace, heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  if (!Q || !K || !V || !O || !delta || !tau || !workspace || !state_ok(st)) return HEART_ERR_INVALID;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return HEART_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  Workspace w = carve(g, workspace);
+  g_launches = 0;
+  cudaError_t e;
+  if (g.flags & HEART_FORCE_DENSE) {
+    fill_dense_outputs_kernel<<<(g.R + 127) / 128, 128, 0, s>>>(g.R, drift_out, refresh_out, w.refresh);
+    ++g_launches;
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "fill_dense_outputs");
+    e = launch_attention(g, Q, K, V, nullptr, nullptr, true, O, lse, w.status, s, &g_launches);
+    if (e != cudaSuccess) return cuda_fail(e, "attention");
+    return HEART_OK;
+  }
+  e = launch_block_sums(g, Q, K, w.bsum, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "block_sums");
+  e = launch_decide(g, w, delta, *st, drift_out, refresh_out, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "decide");
+  e = launch_predict_mask(g, w, tau, w.refresh, *st, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
+  e = launch_attention(g, Q, K, V, st->kv_idx, st->kv_cnt, false, O, lse, w.status, s, &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "attention");
+  return HEART_OK;
+}
+
+int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_host, const void *V_host,
+                    const double *delta, const double *tau, heart_state *st, void *O_host,
+                    double *drift_host, uint8_t *refresh_host, void *Q_dev, void *K_dev, void *V_dev,
+                    void *O_dev, void *workspace, heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  if (cfg->stride_b != 0 || cfg->stride_h != 0 || cfg->stride_n != 0) return HEART_ERR_INVALID;
+  if (!Q_host || !K_host || !V_host || !O_host || !Q_dev || !K_dev || !V_dev || !O_dev || !delta || !tau ||
+      !workspace || !state_ok(st))
+    return HEART_ERR_INVALID;
+  if (!aligned16(Q_dev) || !aligned16(K_dev) || !aligned16(V_dev) || !aligned16(O_dev) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return HEART_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  Workspace w = carve(g, workspace);
+  const size_t bytes = sizeof(uint16_t) * (size_t)g.R * g.N * kD;
+  cudaError_t e = cudaMemcpyAsync(Q_dev, Q_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(K_dev, K_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(V_dev, V_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (host to device)");
+  rc = heart_step(cfg, Q_dev, K_dev, V_dev, delta, tau, st, O_dev, nullptr, w.drift, nullptr, workspace, stream);
+  if (rc != HEART_OK) return rc;
+  e = cudaMemcpyAsync(O_host, O_dev, bytes, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess && drift_host)
+    e = cudaMemcpyAsync(drift_host, w.drift, sizeof(double) * (size_t)g.R, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess && refresh_host)
+    e = cudaMemcpyAsync(refresh_host, w.refresh, (size_t)g.R, cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (device to host)");
+  return HEART_OK;
+}
+
+int heart_get_status(void *workspace, heart_stream_t stream, int32_t *code_out) {
+  if (!workspace || !code_out) return HEART_ERR_INVALID;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t words[2] = {0, 0};
+  cudaError_t e = cudaMemcpyAsync(words, workspace, sizeof words, cudaMemcpyDeviceToHost, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(e, "heart_get_status");
+  *code_out = words[0];
+  if (words[0] != 0) {
+    e = cudaMemsetAsync(workspace, 0, sizeof words, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e, "heart_get_status");
+  }
+  return HEART_OK;
+}
+
+const char *heart_strerror(int code) {
+  switch (code) {
+    case HEART_OK: return "ok";
+    case HEART_ERR_INVALID: return "invalid argument (null pointer, size, stride or alignment)";
+    case HEART_ERR_UNSUPPORTED: return "unsupported shape (head_dim must be 128, block 64 or 128, at most 1024 blocks)";
+    case HEART_ERR_CUDA: return g_errbuf[0] ? g_errbuf : "CUDA error";
+    case HEART_ERR_DEVICE_CHECK: return "device-side check failed (index-list entry out of range or a bounded wait ran out)";
+    default: return "unknown code";
+  }
+}
+
+int heart_last_launch_count(void) { return g_launches; }
+
+}  // extern "C"

@@ -1,0 +1,213 @@
+// Block-importance mask prediction for the refreshed heads (Observation II: rank candidate blocks by
+// importance, retain until the accumulated importance reaches the head's threshold; the minimal
+// cumulative-mass set of Observation I).  Importance = row softmax of the block-pooled Q.K^T scores.
+//
+// One CTA owns TI = 16 query blocks of one head.  Phase 1 is a register-tiled fp64 contraction of
+// the pooled means (each thread 4 query blocks x 4 key blocks, key means staged through shared
+// memory 256 blocks x 32 dims at a time) into a shared-memory tile of scores.  Phase 2 gives each
+// warp two rows: two-pass softmax, then top-p WITHOUT a sort: the kept set is {p > theta} plus the
+// lowest-index ties at theta, where theta is the largest element value whose ">= theta" mass still
+// reaches tau -- found by a 62-step bit-wise search over the IEEE-754 pattern of p (positive
+// doubles order like their bit patterns).  Everything is fp64 so the integer outputs (bit mask,
+// ascending index list, count) agree with a plain fp64 sort-and-accumulate reference except when
+// the cumulative mass is within rounding (1e-15) of tau.
+#include "common.cuh"
+
+namespace heart {
+
+constexpr int TI = 16;    // query blocks per CTA
+constexpr int TJ = 256;   // key blocks per staged pass
+constexpr int TD = 32;    // dims per staged chunk
+constexpr int KLD = TD + 1;
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;  // identical in every lane (each level adds the same two numbers in both partners)
+}
+__device__ __forceinline__ double warp_max(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+template <int NJ>  // NJ*32 >= n_b
+__global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restrict__ bsum, int R, int N,
+                                                           int block, int nb, double scale,
+                                                           const double *__restrict__ tau,
+                                                           const uint8_t *__restrict__ refresh,
+                                                           unsigned flags, uint32_t *__restrict__ mask_bits,
+                                                           int32_t *__restrict__ kv_idx,
+                                                           int32_t *__restrict__ kv_cnt, int idx_stride,
+                                                           int W) {
+  constexpr int NBP = NJ * 32;
+  const int r = blockIdx.y;
+  if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: mask untouched
+  const int I0 = blockIdx.x * TI;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double *S = reinterpret_cast<double *>(smem_raw);  // [TI][NBP]
+  double *Qs = S + TI * NBP;                         // [TI][kD]
+  double *Ks = Qs + TI * kD;                         // [TJ][KLD]
+  const double *bq = bsum + ((size_t)r * nb) * kD;
+  const double *bk = bsum + (((size_t)R + r) * nb) * kD;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int last_cnt = N - (nb - 1) * block;
+
+  for (int e = tid; e < TI * kD; e += 256) {
+    const int i = e / kD, I = I0 + i;
+    double v = 0.0;
+    if (I < nb) v = bq[(size_t)I * kD + (e % kD)] / (double)(I == nb - 1 ? last_cnt : block);
+    Qs[e] = v;
+  }
+
+  // ---- phase 1: S[i][J] = scale * <Qp[I0+i], Kp[J]>
+  const int ig = warp & 3, jh = warp >> 2;
+  for (int jc = 0; jc < nb; jc += TJ) {
+    double acc[4][4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int m = 0; m < 4; ++m) acc[a][m] = 0.0;
+    for (int dc = 0; dc < kD; dc += TD) {
+      __syncthreads();
+#pragma unroll 4
+      for (int k = 0; k < (TJ * TD) / 256; ++k) {
+        const int e = tid + 256 * k, row = e / TD, dd = e % TD, J = jc + row;
+        double v = 0.0;
+        if (J < nb) v = bk[(size_t)J * kD + dc + dd] / (double)(J == nb - 1 ? last_cnt : block);
+        Ks[row * KLD + dd] = v;
+      }
+      __syncthreads();
+#pragma unroll 8
+      for (int dd = 0; dd < TD; ++dd) {
+        double q[4], k[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) q[a] = Qs[(ig * 4 + a) * kD + dc + dd];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) k[m] = Ks[(jh * 128 + lane + 32 * m) * KLD + dd];
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int m = 0; m < 4; ++m) acc[a][m] = fma(q[a], k[m], acc[a][m]);
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int m = 0; m < 4; ++m) {
+        const int J = jc + jh * 128 + lane + 32 * m;
+        if (J < NBP) S[(ig * 4 + a) * NBP + J] = acc[a][m] * scale;
+      }
+  }
+  __syncthreads();
+
+  // ---- phase 2: per-row softmax and top-p; warp w owns rows 2w and 2w+1
+  const unsigned lt_mask = (1u << lane) - 1u;
+  for (int i = warp * 2; i < warp * 2 + 2; ++i) {
+    const int I = I0 + i;
+    if (I >= nb) continue;
+    const size_t row = (size_t)r * nb + I;
+    double p[NJ];
+    const double neg_inf = __longlong_as_double(0xfff0000000000000LL);
+    double mx = neg_inf;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+      const int J = j * 32 + lane;
+      p[j] = (J < nb) ? S[i * NBP + J] : neg_inf;
+      mx = fmax(mx, p[j]);
+    }
+    mx = warp_max(mx);
+    double z = 0.0;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+      const int J = j * 32 + lane;
+      p[j] = (J < nb) ? exp(p[j] - mx) : 0.0;
+      z += p[j];
+    }
+    z = warp_sum(z);
+    double total = 0.0;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+      p[j] = p[j] / z;
+      total += p[j];
+    }
+    total = warp_sum(total);
+
+    const double t = (flags & HEART_FORCE_DENSE) ? 1.0 : tau[r];
+    const bool keep_all = !(t < 1.0) || !(total >= t);
+    long long theta = 0;
+    int m_ties = 0;
+    if (!keep_all) {
+      for (int bit = 61; bit >= 0; --bit) {
+        const long long cand = theta | (1LL << bit);
+        double g = 0.0;
+#pragma unroll
+        for (int j = 0; j < NJ; ++j)
+          if (__double_as_longlong(p[j]) >= cand) g += p[j];
+        g = warp_sum(g);
+        if (g >= t) theta = cand;
+      }
+      double above = 0.0;
+      int nties = 0;
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+        const long long b = __double_as_longlong(p[j]);
+        if (b > theta) above += p[j];
+        nties += (b == theta && j * 32 + lane < nb) ? 1 : 0;
+      }
+      above = warp_sum(above);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) nties += __shfl_xor_sync(0xffffffffu, nties, o);
+      const double th = __longlong_as_double(theta);
+      double c = above;
+      do {  // ties enter in ascending index order, one at a time, until the mass reaches tau
+        c += th;
+        ++m_ties;
+      } while (c < t && m_ties < nties);
+    }
+
+    int base = 0, tie_seen = 0;
+#pragma unroll
+    for (int j = 0; j < NJ; ++j) {
+      const int J = j * 32 + lane;
+      const long long b = __double_as_longlong(p[j]);
+      const bool valid = J < nb;
+      const bool is_tie = valid && !keep_all && b == theta;
+      const unsigned tie_ballot = __ballot_sync(0xffffffffu, is_tie);
+      const int tie_rank = tie_seen + __popc(tie_ballot & lt_mask);
+      tie_seen += __popc(tie_ballot);
+      const bool keep = valid && (keep_all || b > theta || (is_tie && tie_rank < m_ties));
+      const unsigned word = __ballot_sync(0xffffffffu, keep);
+      if (lane == 0 && j < W) mask_bits[row * W + j] = word;
+      if (keep) kv_idx[row * idx_stride + base + __popc(word & lt_mask)] = J;
+      base += __popc(word);
+    }
+    if (lane == 0) kv_cnt[row] = base;
+  }
+}
+
+template <int NJ>
+static cudaError_t launch_nj(const Geom &g, const Workspace &w, const double *tau, const uint8_t *refresh,
+                             heart_state st, cudaStream_t s) {
+  const size_t smem = sizeof(double) * ((size_t)TI * NJ * 32 + TI * kD + TJ * KLD);
+  cudaError_t e = cudaFuncSetAttribute(predict_mask_kernel<NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid((g.nb + TI - 1) / TI, g.R);
+  predict_mask_kernel<NJ><<<grid, 256, smem, s>>>(w.bsum, g.R, g.N, g.block, g.nb, g.scale, tau, refresh,
+                                                 g.flags, st.mask_bits, st.kv_idx, st.kv_cnt,
+                                                 g.idx_stride, g.W);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
+                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches) {
+  ++*launches;
+  const int nj = (g.nb + 31) / 32;
+  if (nj <= 8) return launch_nj<8>(g, w, tau, refresh, st, s);
+  if (nj <= 16) return launch_nj<16>(g, w, tau, refresh, st, s);
+  if (nj <= 24) return launch_nj<24>(g, w, tau, refresh, st, s);
+  return launch_nj<32>(g, w, tau, refresh, st, s);
+}
+
+}  // namespace heart

@@ -1,0 +1,182 @@
+// Streaming statistics of one layer-step: per-block sums of Q and K in a single pass over HBM
+// (token-mean pooling of Algorithm 1 line 1 and the block pooling of the mask predictor share the
+// pass), then the mean-pooled L1 drift, the refresh-or-reuse decision, the layer gate and the
+// anchor update (Eq. mean-pooled drift; Algorithm 1; layer-level gating of the TMR section).
+//
+// Numerics: each thread adds at most block/16 (4 or 8) bf16 values in fp32 -- exact unless an
+// addend lies more than 2^16 below the running sum -- and everything after that (the 16-way
+// combine inside the CTA, the sum over blocks, means, drift) is fp64 in a fixed order, so the
+// result is bit-reproducible run to run: identical inputs give a drift of exactly 0.
+#include "common.cuh"
+
+namespace heart {
+
+__device__ __forceinline__ uint4 ldg_nc_v4(const void *p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// One CTA per (block I, head row r, tensor z).  256 threads: 16 row groups x 16 chunks of 8 dims.
+// Every thread issues all of its 128-bit loads before the first add (block/16 loads in flight).
+template <int BLOCK>
+__global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restrict__ Q,
+                                                         const uint16_t *__restrict__ K, long long sb,
+                                                         long long sh, long long sn, int H, int N,
+                                                         int nb, double *__restrict__ bsum) {
+  constexpr int ITERS = BLOCK / 16;
+  const int I = blockIdx.x, r = blockIdx.y, z = blockIdx.z;
+  const int c = threadIdx.x & 15, g = threadIdx.x >> 4;
+  const uint16_t *X = (z ? K : Q) + (long long)(r / H) * sb + (long long)(r % H) * sh +
+                      (long long)I * BLOCK * sn + c * 8;
+  const int rows = min(BLOCK, N - I * BLOCK);
+
+  uint4 v[ITERS];
+#pragma unroll
+  for (int it = 0; it < ITERS; ++it) {
+    const int row = it * 16 + g;
+    v[it] = (row < rows) ? ldg_nc_v4(X + (long long)row * sn) : make_uint4(0, 0, 0, 0);
+  }
+  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int it = 0; it < ITERS; ++it) {
+    acc[0] += bf16_lo(v[it].x);
+    acc[1] += bf16_hi(v[it].x);
+    acc[2] += bf16_lo(v[it].y);
+    acc[3] += bf16_hi(v[it].y);
+    acc[4] += bf16_lo(v[it].z);
+    acc[5] += bf16_hi(v[it].z);
+    acc[6] += bf16_lo(v[it].w);
+    acc[7] += bf16_hi(v[it].w);
+  }
+  __shared__ double sm[16][kD];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) sm[g][c * 8 + e] = (double)acc[e];
+  __syncthreads();
+  if (threadIdx.x < kD) {
+    double s = 0.0;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) s += sm[k][threadIdx.x];
+    bsum[(((size_t)z * gridDim.y + r) * nb + I) * kD + threadIdx.x] = s;
+  }
+}
+
+// One CTA per (head row r, tensor z), 1024 threads = 8 block ranges x 128 dims.
+// mean[z][r][d] = (sum over blocks, ascending) / N;  part[z][r] = sum_d |anchor - mean|.
+__global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restrict__ bsum, int R, int N,
+                                                          int nb, const double *__restrict__ anchor_q,
+                                                          const double *__restrict__ anchor_k,
+                                                          double *__restrict__ mean,
+                                                          double *__restrict__ part) {
+  const int r = blockIdx.x, z = blockIdx.y;
+  const int d = threadIdx.x & (kD - 1), grp = threadIdx.x >> 7;  // 8 groups
+  const int per = (nb + 7) / 8;
+  const int i0 = grp * per, i1 = min(nb, i0 + per);
+  const double *src = bsum + ((size_t)z * R + r) * nb * kD + d;
+  double s = 0.0;
+  for (int i = i0; i < i1; ++i) s += src[(size_t)i * kD];
+  __shared__ double sm[8][kD];
+  __shared__ double red[kD];
+  sm[grp][d] = s;
+  __syncthreads();
+  if (threadIdx.x < kD) {
+    double t = 0.0;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) t += sm[k][d];
+    const double m = t / (double)N;
+    mean[((size_t)z * R + r) * kD + d] = m;
+    const double a = (z ? anchor_k : anchor_q)[(size_t)r * kD + d];
+    red[d] = fabs(a - m);
+  }
+  __syncthreads();
+  for (int w = kD / 2; w > 0; w >>= 1) {  // fixed-shape tree: deterministic
+    if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) part[(size_t)z * R + r] = red[0];
+}
+
+// One CTA per batch entry: head-wise rule, gate over the H heads, anchor update.
+__global__ void __launch_bounds__(128) decide_kernel(int H, int R, const double *__restrict__ part,
+                                                     const double *__restrict__ mean,
+                                                     const double *__restrict__ delta, double gate_lo,
+                                                     double gate_hi, unsigned flags,
+                                                     double *__restrict__ anchor_q,
+                                                     double *__restrict__ anchor_k,
+                                                     uint8_t *__restrict__ has_anchor,
+                                                     uint8_t *__restrict__ refresh_ws,
+                                                     double *__restrict__ drift_out,
+                                                     uint8_t *__restrict__ refresh_out) {
+  extern __shared__ uint8_t sh_flags[];  // [2*H]: decision, had_anchor
+  __shared__ int cnt;
+  const int b = blockIdx.x;
+  if (threadIdx.x == 0) cnt = 0;
+  __syncthreads();
+  for (int h = threadIdx.x; h < H; h += blockDim.x) {
+    const int r = b * H + h;
+    const bool had = has_anchor[r] != 0;
+    const double dr = had ? (part[r] + part[R + r]) : __longlong_as_double(0x7ff0000000000000LL);
+    bool rf = !had || (dr > delta[r]);
+    if (flags & HEART_FORCE_REFRESH) rf = true;
+    sh_flags[h] = rf;
+    sh_flags[H + h] = had;
+    if (drift_out) drift_out[r] = dr;
+    if (rf) atomicAdd(&cnt, 1);
+  }
+  __syncthreads();
+  const double f = (double)cnt / (double)H;
+  for (int h = threadIdx.x; h < H; h += blockDim.x) {
+    bool rf = sh_flags[h];
+    if (f < gate_lo) {
+      if (sh_flags[H + h]) rf = false;
+    } else if (f > gate_hi) {
+      rf = true;
+    }
+    sh_flags[h] = rf;
+    const int r = b * H + h;
+    refresh_ws[r] = rf;
+    if (refresh_out) refresh_out[r] = rf;
+    if (rf) has_anchor[r] = 1;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < H * kD; e += blockDim.x) {
+    const int h = e / kD, r = b * H + h;
+    if (sh_flags[h]) {
+      anchor_q[(size_t)r * kD + (e % kD)] = mean[(size_t)r * kD + (e % kD)];
+      anchor_k[(size_t)r * kD + (e % kD)] = mean[((size_t)R + r) * kD + (e % kD)];
+    }
+  }
+}
+
+cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, double *bsum,
+                              cudaStream_t s, int *launches) {
+  dim3 grid(g.nb, g.R, 2);
+  const uint16_t *q = static_cast<const uint16_t *>(Q), *k = static_cast<const uint16_t *>(K);
+  if (g.block == 64)
+    block_sums_kernel<64><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, bsum);
+  else
+    block_sums_kernel<128><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, bsum);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta, heart_state st,
+                          double *drift_out, uint8_t *refresh_out, cudaStream_t s, int *launches) {
+  mean_drift_kernel<<<dim3(g.R, 2), 1024, 0, s>>>(w.bsum, g.R, g.N, g.nb, st.anchor_q, st.anchor_k,
+                                                  w.mean, w.part);
+  ++*launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  decide_kernel<<<g.B, 128, 2 * g.H, s>>>(g.H, g.R, w.part, w.mean, delta, g.gate_lo, g.gate_hi,
+                                          g.flags, st.anchor_q, st.anchor_k, st.has_anchor, w.refresh,
+                                          drift_out, refresh_out);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace heart

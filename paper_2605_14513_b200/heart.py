@@ -1,0 +1,188 @@
+"""Thin Python binding of the C ABI in include/heart.h (argument marshalling only).
+
+Every step of the hot path runs in the CUDA kernels of libheart.so; torch is used
+for device memory and streams.  Importing this module loads the library and
+fails loudly if it has not been built -- there is no CPU or eager fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libheart.so")
+
+OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_CHECK = 0, 1, 2, 3, 4
+FORCE_REFRESH, FORCE_DENSE = 1, 2
+MAX_BLOCKS = 1024
+
+# Every symbol include/heart.h declares.
+SYMBOLS = (
+    "heart_workspace_bytes", "heart_state_reset", "heart_drift", "heart_predict_mask",
+    "heart_block_sparse_attn", "heart_step", "heart_step_host", "heart_get_status", "heart_strerror",
+    "heart_last_launch_count",
+)
+
+
+class Config(C.Structure):
+    _fields_ = [("B", C.c_int32), ("H", C.c_int32), ("N", C.c_int32), ("D", C.c_int32),
+                ("block", C.c_int32),
+                ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_n", C.c_int64),
+                ("scale", C.c_double), ("gate_lo", C.c_double), ("gate_hi", C.c_double),
+                ("idx_stride", C.c_int32), ("flags", C.c_uint32)]
+
+
+class StateStruct(C.Structure):
+    _fields_ = [("anchor_q", C.c_void_p), ("anchor_k", C.c_void_p), ("has_anchor", C.c_void_p),
+                ("mask_bits", C.c_void_p), ("kv_idx", C.c_void_p), ("kv_cnt", C.c_void_p)]
+
+
+class HeartError(RuntimeError):
+    def __init__(self, code):
+        self.code = code
+        super().__init__(f"heart error {code}: {lib().heart_strerror(code).decode()}")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded libheart.so (raises if it is missing: build it with build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} not found: run `python -m paper_2605_14513_b200.build` "
+                              "(or __graft_entry__.build()) -- there is no fallback path")
+        l = C.CDLL(_LIB_PATH)
+        l.heart_workspace_bytes.restype = C.c_size_t
+        l.heart_workspace_bytes.argtypes = [C.POINTER(Config)]
+        l.heart_strerror.restype = C.c_char_p
+        l.heart_strerror.argtypes = [C.c_int]
+        l.heart_last_launch_count.restype = C.c_int
+        vp = C.c_void_p
+        l.heart_state_reset.argtypes = [C.POINTER(Config), C.POINTER(StateStruct), vp]
+        l.heart_drift.argtypes = [C.POINTER(Config), vp, vp, vp, C.POINTER(StateStruct), vp, vp, vp, vp]
+        l.heart_predict_mask.argtypes = [C.POINTER(Config), vp, vp, vp, vp, C.POINTER(StateStruct), vp, vp]
+        l.heart_block_sparse_attn.argtypes = [C.POINTER(Config), vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        l.heart_step.argtypes = [C.POINTER(Config), vp, vp, vp, vp, vp, C.POINTER(StateStruct), vp, vp, vp, vp, vp, vp]
+        l.heart_step_host.argtypes = [C.POINTER(Config), vp, vp, vp, vp, vp, C.POINTER(StateStruct)] + [vp] * 9
+        l.heart_get_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+        for fn in ("heart_state_reset", "heart_drift", "heart_predict_mask", "heart_block_sparse_attn",
+                   "heart_step", "heart_step_host", "heart_get_status"):
+            getattr(l, fn).restype = C.c_int
+        _lib = l
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc):
+    if rc != OK:
+        raise HeartError(rc)
+
+
+def n_blocks(N, block):
+    return (N + block - 1) // block
+
+
+def make_config(B, H, N, block, D=128, scale=0.0, gate_lo=0.0, gate_hi=1.0, idx_stride=None, flags=0,
+                strides=(0, 0, 0)) -> Config:
+    nb = n_blocks(N, block)
+    return Config(B, H, N, D, block, strides[0], strides[1], strides[2], scale, gate_lo, gate_hi,
+                  idx_stride if idx_stride is not None else nb, flags)
+
+
+def config_for(x: torch.Tensor, block, **kw) -> Config:
+    """Config for a [B, H, N, D] bf16 tensor (strides taken from the tensor)."""
+    assert x.dim() == 4 and x.dtype == torch.bfloat16 and x.stride(3) == 1
+    B, H, N, D = x.shape
+    return make_config(B, H, N, block, D=D, strides=(x.stride(0), x.stride(1), x.stride(2)), **kw)
+
+
+class State:
+    """Caller-owned TMR state of one layer (device tensors + the C struct that points at them)."""
+
+    def __init__(self, cfg: Config, device="cuda"):
+        R, nb = cfg.B * cfg.H, n_blocks(cfg.N, cfg.block)
+        self.R, self.nb, self.W = R, nb, (nb + 31) // 32
+        self.anchor_q = torch.zeros((R, cfg.D), dtype=torch.float64, device=device)
+        self.anchor_k = torch.zeros((R, cfg.D), dtype=torch.float64, device=device)
+        self.has_anchor = torch.zeros(R, dtype=torch.uint8, device=device)
+        self.mask_bits = torch.zeros((R, nb, self.W), dtype=torch.int32, device=device)
+        self.kv_idx = torch.full((R, nb, cfg.idx_stride), -1, dtype=torch.int32, device=device)
+        self.kv_cnt = torch.zeros((R, nb), dtype=torch.int32, device=device)
+        self.struct = StateStruct(*(t.data_ptr() for t in self.tensors()))
+
+    def tensors(self):
+        return (self.anchor_q, self.anchor_k, self.has_anchor, self.mask_bits, self.kv_idx, self.kv_cnt)
+
+    def state_dict(self):
+        return {k: getattr(self, k).clone() for k in ("anchor_q", "anchor_k", "has_anchor", "mask_bits", "kv_idx", "kv_cnt")}
+
+    def load_state_dict(self, d):
+        for k, v in d.items():
+            getattr(self, k).copy_(v)
+
+
+def workspace_bytes(cfg: Config) -> int:
+    return int(lib().heart_workspace_bytes(C.byref(cfg)))
+
+
+def new_workspace(cfg: Config, device="cuda") -> torch.Tensor:
+    n = workspace_bytes(cfg)
+    if n == 0:
+        raise HeartError(ERR_UNSUPPORTED)
+    return torch.zeros(n, dtype=torch.uint8, device=device)
+
+
+def heart_state_reset(cfg, st: State):
+    _check(lib().heart_state_reset(C.byref(cfg), C.byref(st.struct), _stream()))
+
+
+def heart_drift(cfg, Q, K, delta, st: State, ws, drift_out=None, refresh_out=None):
+    _check(lib().heart_drift(C.byref(cfg), _ptr(Q), _ptr(K), _ptr(delta), C.byref(st.struct), _ptr(drift_out),
+                             _ptr(refresh_out), _ptr(ws), _stream()))
+
+
+def heart_predict_mask(cfg, Q, K, tau, st: State, ws, refresh=None):
+    _check(lib().heart_predict_mask(C.byref(cfg), _ptr(Q), _ptr(K), _ptr(tau), _ptr(refresh), C.byref(st.struct),
+                                    _ptr(ws), _stream()))
+
+
+def heart_block_sparse_attn(cfg, Q, K, V, kv_idx, kv_cnt, O, ws, lse=None):
+    _check(lib().heart_block_sparse_attn(C.byref(cfg), _ptr(Q), _ptr(K), _ptr(V), _ptr(kv_idx), _ptr(kv_cnt),
+                                         _ptr(O), _ptr(lse), _ptr(ws), _stream()))
+
+
+def heart_step(cfg, Q, K, V, delta, tau, st: State, O, ws, lse=None, drift_out=None, refresh_out=None):
+    _check(lib().heart_step(C.byref(cfg), _ptr(Q), _ptr(K), _ptr(V), _ptr(delta), _ptr(tau), C.byref(st.struct),
+                            _ptr(O), _ptr(lse), _ptr(drift_out), _ptr(refresh_out), _ptr(ws), _stream()))
+
+
+def heart_step_host(cfg, Qh, Kh, Vh, delta, tau, st: State, Oh, staging, ws, drift_host=None, refresh_host=None):
+    """Host-buffer step: Qh/Kh/Vh/Oh (and the optional drift/refresh) are CPU tensors, ideally pinned;
+    `staging` = (Q_dev, K_dev, V_dev, O_dev) device tensors.  Asynchronous on the current stream."""
+    for t in (Qh, Kh, Vh, Oh):
+        assert t.device.type == "cpu" and t.is_contiguous()
+    _check(lib().heart_step_host(C.byref(cfg), _ptr(Qh), _ptr(Kh), _ptr(Vh), _ptr(delta), _ptr(tau),
+                                 C.byref(st.struct), _ptr(Oh), _ptr(drift_host), _ptr(refresh_host),
+                                 _ptr(staging[0]), _ptr(staging[1]), _ptr(staging[2]), _ptr(staging[3]), _ptr(ws),
+                                 _stream()))
+
+
+def heart_get_status(ws) -> int:
+    code = C.c_int32(0)
+    _check(lib().heart_get_status(_ptr(ws), _stream(), C.byref(code)))
+    return code.value
+
+
+def heart_last_launch_count() -> int:
+    return int(lib().heart_last_launch_count())
