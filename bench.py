@@ -38,7 +38,7 @@ def parse():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="wan1.3b-480p")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cpu-sample-rows", type=int, default=8, help="query blocks the CPU oracle attends per step")
+    ap.add_argument("--cpu-sample-rows", type=int, default=64, help="query blocks the CPU oracle attends per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -330,7 +330,7 @@ def cpu_baseline(args, wl, steps_in, W):
     ost = oracle.State(wl.B, wl.H, wl.N, wl.D, wl.block)
     rs = np.random.RandomState(0)
     est, spent, n = [], 0.0, 0
-    budget = 25.0
+    budget = 20.0
     # step 0 builds the anchors and masks (all heads refresh); later steps show the steady mix
     for t in range(min(len(steps_in), W + 3)):
         Qb, Kb, Vb = (inputs.bits(x) for x in steps_in[t])
