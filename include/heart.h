@@ -46,8 +46,10 @@ enum {
   HEART_ERR_INVALID = 1,      /* null pointer, bad size/stride/alignment               */
   HEART_ERR_UNSUPPORTED = 2,  /* D != 128, block not in {64,128}, n_b > 1024            */
   HEART_ERR_CUDA = 3,         /* a CUDA call or launch failed (see heart_strerror)      */
-  HEART_ERR_DEVICE_CHECK = 4  /* a device-side check failed: bad index-list entry or a  */
+  HEART_ERR_DEVICE_CHECK = 4, /* a device-side check failed: bad index-list entry or a  */
                               /* bounded wait ran out; only via heart_get_status        */
+  HEART_ERR_TOO_LARGE = 5     /* heart_drift_static: the shape needs more scratch than   */
+                              /* HEART_STATIC_SCRATCH_BYTES                              */
 };
 
 #define HEART_FORCE_REFRESH 1u /* every head refreshes this step (decision overridden)  */
@@ -140,6 +142,37 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
                     const double *delta, const double *tau, heart_state *st, void *O_host,
                     double *drift_host, uint8_t *refresh_host, void *Q_dev, void *K_dev, void *V_dev,
                     void *O_dev, void *workspace, heart_stream_t stream);
+
+/* Built-in scratch of heart_drift_static: 16 MiB, enough for B*H*n_b <= ~8100 head-row blocks
+ * (e.g. 12 heads x 512 blocks; the 40-head and 720P shapes need the caller-allocated path). */
+#define HEART_STATIC_SCRATCH_BYTES (16u << 20)
+
+/* heart_drift without a workspace argument, for callers that cannot allocate device memory.
+ * (No counterpart in the paper: this is a packaging variant of call (a) above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a host framework's
+ * allocator-managed region where foreign allocations are forbidden or would fragment a fully
+ * reserved GPU, in a real-time or callback context that must not block on the driver's allocator,
+ * or a plugin that is handed Q/K and the TMR state but no way to obtain scratch.  Such a caller
+ * still passes its inputs, outputs and state; only the scratch (block sums, means, flags) comes
+ * from a fixed HEART_STATIC_SCRATCH_BYTES array compiled into the library.  The call makes no
+ * cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * Same arguments, results and error codes as heart_drift, except:
+ *   - no `workspace`; st->mask_bits / kv_idx / kv_cnt may be NULL (they are not touched);
+ *   - a shape whose heart_workspace_bytes exceeds HEART_STATIC_SCRATCH_BYTES is rejected with
+ *     HEART_ERR_TOO_LARGE before anything is launched;
+ *   - the per-block sums it leaves behind are in the built-in array, not in a caller workspace,
+ *     so a following heart_predict_mask recomputes them (it always does).
+ * The array is part of the library image: every GPU that loads the library holds those 16 MiB
+ * until the process exits.  The first call on each device looks the array's device address up
+ * (with that device current) and caches it; make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents: every
+ * value the kernels read from it is rewritten by the same call first, so nothing needs clearing,
+ * but two calls that overlap on the GPU (different streams, no ordering between them) race on it
+ * and give undefined results -- serialise them. */
+int heart_drift_static(const heart_config *cfg, const void *Q, const void *K, const double *delta,
+                       heart_state *st, double *drift_out, uint8_t *refresh_out, heart_stream_t stream);
 
 /* Synchronises `stream`, reads the workspace status word into *code_out (host) and clears it.
  * The only call that blocks. */

@@ -14,7 +14,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libheart.so")
 
-OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_CHECK = 0, 1, 2, 3, 4
+OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
+STATIC_SCRATCH_BYTES = 16 << 20
 FORCE_REFRESH, FORCE_DENSE = 1, 2
 MAX_BLOCKS = 1024
 
@@ -22,7 +23,7 @@ MAX_BLOCKS = 1024
 SYMBOLS = (
     "heart_workspace_bytes", "heart_state_reset", "heart_drift", "heart_predict_mask",
     "heart_block_sparse_attn", "heart_step", "heart_step_host", "heart_get_status", "heart_strerror",
-    "heart_last_launch_count",
+    "heart_last_launch_count", "heart_drift_static",
 )
 
 
@@ -69,6 +70,8 @@ def lib():
         l.heart_step.argtypes = [C.POINTER(Config), vp, vp, vp, vp, vp, C.POINTER(StateStruct), vp, vp, vp, vp, vp, vp]
         l.heart_step_host.argtypes = [C.POINTER(Config), vp, vp, vp, vp, vp, C.POINTER(StateStruct)] + [vp] * 9
         l.heart_get_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
+        l.heart_drift_static.argtypes = [C.POINTER(Config), vp, vp, vp, C.POINTER(StateStruct), vp, vp, vp]
+        l.heart_drift_static.restype = C.c_int
         for fn in ("heart_state_reset", "heart_drift", "heart_predict_mask", "heart_block_sparse_attn",
                    "heart_step", "heart_step_host", "heart_get_status"):
             getattr(l, fn).restype = C.c_int
@@ -176,6 +179,13 @@ def heart_step_host(cfg, Qh, Kh, Vh, delta, tau, st: State, Oh, staging, ws, dri
                                  C.byref(st.struct), _ptr(Oh), _ptr(drift_host), _ptr(refresh_host),
                                  _ptr(staging[0]), _ptr(staging[1]), _ptr(staging[2]), _ptr(staging[3]), _ptr(ws),
                                  _stream()))
+
+
+def heart_drift_static(cfg, Q, K, delta, st: State, drift_out=None, refresh_out=None):
+    """heart_drift for callers that cannot allocate: scratch comes from the library's built-in
+    16 MiB array (shapes that need more raise ERR_TOO_LARGE).  Calls on one device must not overlap."""
+    _check(lib().heart_drift_static(C.byref(cfg), _ptr(Q), _ptr(K), _ptr(delta), C.byref(st.struct),
+                                    _ptr(drift_out), _ptr(refresh_out), _stream()))
 
 
 def heart_get_status(ws) -> int:
