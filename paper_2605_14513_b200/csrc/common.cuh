@@ -15,12 +15,25 @@ struct Geom {
   long long sb, sh, sn;  // element strides of Q/K/V/O
   double scale, gate_lo, gate_hi;
   unsigned flags;
+  int bpc, nchunks;  // block-sum kernel: key/query blocks per CTA and CTAs per (head row, tensor)
 };
+
+// Chunking of the block-sum pass: about 8 CTAs per SM on a 148-SM part, whatever the device (the
+// split fixes the summation order, so it must depend on the shape only).
+__host__ inline void set_chunks(Geom &g) {
+  const int target = 148 * 8;
+  int per_pair = (target + 2 * g.R - 1) / (2 * g.R);
+  if (per_pair < 1) per_pair = 1;
+  g.bpc = (g.nb + per_pair - 1) / per_pair;
+  if (g.bpc < 1) g.bpc = 1;
+  g.nchunks = (g.nb + g.bpc - 1) / g.bpc;
+}
 
 // Workspace layout (all offsets 256-byte aligned).
 struct Workspace {
   int32_t *status;    // [64]   word 0: sticky device-check code; word 1: detail
   double *bsum;       // [2][R][nb][D]  per-block sums of Q (0) and K (1)
+  double *psum;       // [2][R][nchunks][D]  per-CTA partial token sums
   double *mean;       // [2][R][D]      token means of the current step
   double *part;       // [2][R]         L1 parts of the drift
   uint8_t *pre;       // [R]            head-wise decision before the gate
@@ -39,6 +52,8 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   off += align256(64 * sizeof(int32_t));
   w.bsum = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * 2 * (size_t)g.R * g.nb * kD);
+  w.psum = reinterpret_cast<double *>(p + off);
+  off += align256(sizeof(double) * 2 * (size_t)g.R * g.nchunks * kD);
   w.mean = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * 2 * (size_t)g.R * kD);
   w.part = reinterpret_cast<double *>(p + off);
@@ -55,7 +70,7 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
 
 // Launchers (defined in the kernel files). Each returns the cudaError_t of its launches and
 // adds the number of kernels it launched to *launches.
-cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, double *bsum,
+cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, const Workspace &w,
                               cudaStream_t s, int *launches);
 cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta, heart_state st,
                           double *drift_out, uint8_t *refresh_out, cudaStream_t s, int *launches);

@@ -52,6 +52,7 @@ int make_geom(const heart_config *c, Geom *g) {
   g->gate_hi = c->gate_hi;
   if (isnan(g->gate_lo) || isnan(g->gate_hi)) return HEART_ERR_INVALID;
   g->flags = c->flags;
+  set_chunks(*g);
   return HEART_OK;
 }
 
@@ -102,7 +103,7 @@ int heart_drift(const heart_config *cfg, const void *Q, const void *K, const dou
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   Workspace w = carve(g, workspace);
   g_launches = 0;
-  cudaError_t e = launch_block_sums(g, Q, K, w.bsum, s, &g_launches);
+  cudaError_t e = launch_block_sums(g, Q, K, w, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "block_sums");
   e = launch_decide(g, w, delta, *st, drift_out, refresh_out, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "decide");
@@ -119,7 +120,7 @@ int heart_predict_mask(const heart_config *cfg, const void *Q, const void *K, co
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   Workspace w = carve(g, workspace);
   g_launches = 0;
-  cudaError_t e = launch_block_sums(g, Q, K, w.bsum, s, &g_launches);
+  cudaError_t e = launch_block_sums(g, Q, K, w, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "block_sums");
   e = launch_predict_mask(g, w, tau, refresh, *st, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
@@ -168,7 +169,7 @@ int heart_step(const heart_config *cfg, const void *Q, const void *K, const void
     if (e != cudaSuccess) return cuda_fail(e, "attention");
     return HEART_OK;
   }
-  e = launch_block_sums(g, Q, K, w.bsum, s, &g_launches);
+  e = launch_block_sums(g, Q, K, w, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "block_sums");
   e = launch_decide(g, w, delta, *st, drift_out, refresh_out, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "decide");

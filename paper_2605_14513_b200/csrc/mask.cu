@@ -52,11 +52,12 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
   const double *bk = bsum + (((size_t)R + r) * nb) * kD;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int last_cnt = N - (nb - 1) * block;
+  const double inv_block = 1.0 / (double)block;
 
   for (int e = tid; e < TI * kD; e += 256) {
     const int i = e / kD, I = I0 + i;
     double v = 0.0;
-    if (I < nb) v = bq[(size_t)I * kD + (e % kD)] / (double)(I == nb - 1 ? last_cnt : block);
+    if (I < nb) v = (I == nb - 1) ? bq[(size_t)I * kD + (e % kD)] / (double)last_cnt : bq[(size_t)I * kD + (e % kD)] * inv_block;
     Qs[e] = v;
   }
 
@@ -70,12 +71,19 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
       for (int m = 0; m < 4; ++m) acc[a][m] = 0.0;
     for (int dc = 0; dc < kD; dc += TD) {
       __syncthreads();
-#pragma unroll 4
-      for (int k = 0; k < (TJ * TD) / 256; ++k) {
-        const int e = tid + 256 * k, row = e / TD, dd = e % TD, J = jc + row;
-        double v = 0.0;
-        if (J < nb) v = bk[(size_t)J * kD + dc + dd] / (double)(J == nb - 1 ? last_cnt : block);
-        Ks[row * KLD + dd] = v;
+      {  // all 32 loads of this thread in flight before the first use
+        double v[(TJ * TD) / 256];
+#pragma unroll
+        for (int k = 0; k < (TJ * TD) / 256; ++k) {
+          const int e = tid + 256 * k, J = jc + e / TD;
+          v[k] = (J < nb) ? bk[(size_t)J * kD + dc + (e % TD)] : 0.0;
+        }
+#pragma unroll
+        for (int k = 0; k < (TJ * TD) / 256; ++k) {
+          const int e = tid + 256 * k, row = e / TD, J = jc + row;
+          // full blocks: 1/block is a power of two, so the product equals the division exactly
+          Ks[row * KLD + (e % TD)] = (J == nb - 1) ? v[k] / (double)last_cnt : v[k] * inv_block;
+        }
       }
       __syncthreads();
 #pragma unroll 8

@@ -5,8 +5,9 @@
 //
 // Numerics: each thread adds at most block/16 (4 or 8) bf16 values in fp32 -- exact unless an
 // addend lies more than 2^16 below the running sum -- and everything after that (the 16-way
-// combine inside the CTA, the sum over blocks, means, drift) is fp64 in a fixed order, so the
-// result is bit-reproducible run to run: identical inputs give a drift of exactly 0.
+// combine inside the CTA, the sum over the CTA's blocks, the sum over CTAs, means, drift) is fp64 in
+// an order fixed by the shape alone, so the result is bit-reproducible run to run: identical inputs
+// give a drift of exactly 0.
 #include "common.cuh"
 
 namespace heart {
@@ -22,63 +23,79 @@ __device__ __forceinline__ uint4 ldg_nc_v4(const void *p) {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// One CTA per (block I, head row r, tensor z).  256 threads: 16 row groups x 16 chunks of 8 dims.
-// Every thread issues all of its 128-bit loads before the first add (block/16 loads in flight).
+// One CTA per (chunk of consecutive blocks, head row r, tensor z).  256 threads: 16 row groups x 16
+// chunks of 8 dims.  The 128-bit loads of block i+1 are issued before block i is reduced, so every
+// thread keeps BLOCK/16 loads in flight across the shared-memory combine.
 template <int BLOCK>
 __global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restrict__ Q,
                                                          const uint16_t *__restrict__ K, long long sb,
                                                          long long sh, long long sn, int H, int N,
-                                                         int nb, double *__restrict__ bsum) {
+                                                         int nb, int bpc, double *__restrict__ bsum,
+                                                         double *__restrict__ psum) {
   constexpr int ITERS = BLOCK / 16;
-  const int I = blockIdx.x, r = blockIdx.y, z = blockIdx.z;
+  const int chunk = blockIdx.x, r = blockIdx.y, z = blockIdx.z, R = gridDim.y;
   const int c = threadIdx.x & 15, g = threadIdx.x >> 4;
-  const uint16_t *X = (z ? K : Q) + (long long)(r / H) * sb + (long long)(r % H) * sh +
-                      (long long)I * BLOCK * sn + c * 8;
-  const int rows = min(BLOCK, N - I * BLOCK);
-
-  uint4 v[ITERS];
-#pragma unroll
-  for (int it = 0; it < ITERS; ++it) {
-    const int row = it * 16 + g;
-    v[it] = (row < rows) ? ldg_nc_v4(X + (long long)row * sn) : make_uint4(0, 0, 0, 0);
-  }
-  float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-  for (int it = 0; it < ITERS; ++it) {
-    acc[0] += bf16_lo(v[it].x);
-    acc[1] += bf16_hi(v[it].x);
-    acc[2] += bf16_lo(v[it].y);
-    acc[3] += bf16_hi(v[it].y);
-    acc[4] += bf16_lo(v[it].z);
-    acc[5] += bf16_hi(v[it].z);
-    acc[6] += bf16_lo(v[it].w);
-    acc[7] += bf16_hi(v[it].w);
-  }
+  const uint16_t *X = (z ? K : Q) + (long long)(r / H) * sb + (long long)(r % H) * sh + c * 8;
+  const int i0 = chunk * bpc, i1 = min(nb, i0 + bpc);
   __shared__ double sm[16][kD];
+
+  uint4 cur[ITERS], nxt[ITERS];
+  auto load_block = [&](int I, uint4 (&v)[ITERS]) {
+    const int rows = min(BLOCK, N - I * BLOCK);
+    const uint16_t *base = X + (long long)I * BLOCK * sn;
 #pragma unroll
-  for (int e = 0; e < 8; ++e) sm[g][c * 8 + e] = (double)acc[e];
-  __syncthreads();
-  if (threadIdx.x < kD) {
-    double s = 0.0;
+    for (int it = 0; it < ITERS; ++it) {
+      const int row = it * 16 + g;
+      v[it] = (row < rows) ? ldg_nc_v4(base + (long long)row * sn) : make_uint4(0, 0, 0, 0);
+    }
+  };
+  load_block(i0, cur);
+  double total = 0.0;  // threads 0..127: running token sum of dim threadIdx.x over this CTA's blocks
+  for (int I = i0; I < i1; ++I) {
+    if (I + 1 < i1) load_block(I + 1, nxt);
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int k = 0; k < 16; ++k) s += sm[k][threadIdx.x];
-    bsum[(((size_t)z * gridDim.y + r) * nb + I) * kD + threadIdx.x] = s;
+    for (int it = 0; it < ITERS; ++it) {
+      acc[0] += bf16_lo(cur[it].x);
+      acc[1] += bf16_hi(cur[it].x);
+      acc[2] += bf16_lo(cur[it].y);
+      acc[3] += bf16_hi(cur[it].y);
+      acc[4] += bf16_lo(cur[it].z);
+      acc[5] += bf16_hi(cur[it].z);
+      acc[6] += bf16_lo(cur[it].w);
+      acc[7] += bf16_hi(cur[it].w);
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sm[g][c * 8 + e] = (double)acc[e];
+    __syncthreads();
+    if (threadIdx.x < kD) {
+      double s = 0.0;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) s += sm[k][threadIdx.x];
+      bsum[(((size_t)z * R + r) * nb + I) * kD + threadIdx.x] = s;
+      total += s;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) cur[it] = nxt[it];
   }
+  if (threadIdx.x < kD) psum[(((size_t)z * R + r) * gridDim.x + chunk) * kD + threadIdx.x] = total;
 }
 
-// One CTA per (head row r, tensor z), 1024 threads = 8 block ranges x 128 dims.
-// mean[z][r][d] = (sum over blocks, ascending) / N;  part[z][r] = sum_d |anchor - mean|.
-__global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restrict__ bsum, int R, int N,
-                                                          int nb, const double *__restrict__ anchor_q,
+// One CTA per (head row r, tensor z), 1024 threads = 8 ranges of partial sums x 128 dims.
+// mean[z][r][d] = (sum over the per-CTA partials, ascending) / N;  part[z][r] = sum_d |anchor - mean|.
+__global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restrict__ psum, int R, int N,
+                                                          int nchunks, const double *__restrict__ anchor_q,
                                                           const double *__restrict__ anchor_k,
                                                           double *__restrict__ mean,
                                                           double *__restrict__ part) {
   const int r = blockIdx.x, z = blockIdx.y;
   const int d = threadIdx.x & (kD - 1), grp = threadIdx.x >> 7;  // 8 groups
-  const int per = (nb + 7) / 8;
-  const int i0 = grp * per, i1 = min(nb, i0 + per);
-  const double *src = bsum + ((size_t)z * R + r) * nb * kD + d;
+  const int per = (nchunks + 7) / 8;
+  const int i0 = grp * per, i1 = min(nchunks, i0 + per);
+  const double *src = psum + ((size_t)z * R + r) * nchunks * kD + d;
   double s = 0.0;
+#pragma unroll 8
   for (int i = i0; i < i1; ++i) s += src[(size_t)i * kD];
   __shared__ double sm[8][kD];
   __shared__ double red[kD];
@@ -153,21 +170,21 @@ __global__ void __launch_bounds__(128) decide_kernel(int H, int R, const double 
   }
 }
 
-cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, double *bsum,
+cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, const Workspace &w,
                               cudaStream_t s, int *launches) {
-  dim3 grid(g.nb, g.R, 2);
+  dim3 grid(g.nchunks, g.R, 2);
   const uint16_t *q = static_cast<const uint16_t *>(Q), *k = static_cast<const uint16_t *>(K);
   if (g.block == 64)
-    block_sums_kernel<64><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, bsum);
+    block_sums_kernel<64><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bsum, w.psum);
   else
-    block_sums_kernel<128><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, bsum);
+    block_sums_kernel<128><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bsum, w.psum);
   ++*launches;
   return cudaGetLastError();
 }
 
 cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta, heart_state st,
                           double *drift_out, uint8_t *refresh_out, cudaStream_t s, int *launches) {
-  mean_drift_kernel<<<dim3(g.R, 2), 1024, 0, s>>>(w.bsum, g.R, g.N, g.nb, st.anchor_q, st.anchor_k,
+  mean_drift_kernel<<<dim3(g.R, 2), 1024, 0, s>>>(w.psum, g.R, g.N, g.nchunks, st.anchor_q, st.anchor_k,
                                                   w.mean, w.part);
   ++*launches;
   cudaError_t e = cudaGetLastError();
