@@ -7,15 +7,19 @@
 // entry carries one flag bit per query block.  K/V blocks are fetched once per CTA and shared by
 // both tiles; a tile skips the MMAs of union entries none of its query blocks lists.
 //
-// Warp roles (384 threads):
+// Warp roles (320 threads):
 //   warp 0      TMA producer: Q tiles once, then the listed K and V blocks through shared-memory
 //               rings (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers).
 //   warp 1      MMA issuer (one lane): S_t = Q_t K^T into tensor memory (tcgen05.mma, operands in
 //               shared memory), O_t += P_t V with P_t read from tensor memory; the two tiles are
 //               interleaved so one tile's softmax overlaps the other tile's MMAs.
-//   warps 4-7   softmax of tile 0, warps 8-11 softmax of tile 1: thread = query row; reads its S
-//               row from tensor memory, keeps the running max / sum, writes P (bf16) back over S,
-//               rescales O only when the max grew by more than 2^8, and writes O / lse at the end.
+//   warps 2-9   softmax: both warpgroups work on the tile whose scores are ready, warpgroup a on key
+//               columns [64a, 64a+64); thread = (query row, column half).  It reads its half of the S
+//               row from tensor memory, the two halves exchange their row maxima through shared
+//               memory, it keeps the running max / partial sum, writes P (bf16) back over S,
+//               rescales its half of O only when the max grew by more than 2^8, and writes its half
+//               of O (and lse) at the end.  Two warps per scheduler work at the same time, so the
+//               exponentials (MUFU) of one overlap the FMA/ALU work of the other.
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P_t aliases S_t.
 //
 // Every wait is bounded; a wait that runs out raises a CTA-wide abort flag and the status word, the
@@ -28,29 +32,32 @@
 namespace heart {
 using namespace tc;
 
-constexpr int kAttnThreads = 384;
+constexpr int kAttnThreads = 320;
 constexpr int kMaxNb = HEART_MAX_BLOCKS;
 
-template <int BK>
+// Shared-memory plan.  A key tile always holds 128 keys = SUBS key blocks of B tokens.
+template <int B>
 struct AttnSmem {
-  static constexpr int NQB = 256 / BK;            // query blocks per CTA
-  static constexpr int QBT = 128 / BK;            // query blocks per 128-row tile
-  static constexpr int NS = (BK == 128) ? 2 : 4;  // ring depth of K and of V
-  static constexpr int Q_BYTES = 128 * 256;       // one Q tile  [2 halves][128 rows][64] bf16
-  static constexpr int KV_BYTES = BK * 256;       // one K/V tile [2 halves][BK rows][64] bf16
+  static constexpr int SUBS = 128 / B;       // key blocks per 128-key tile (1 or 2)
+  static constexpr int NQB = 256 / B;        // query blocks per CTA (2 or 4)
+  static constexpr int QBT = 128 / B;        // query blocks per 128-row query tile
+  static constexpr int NS = 2;               // ring depth of K and of V
+  static constexpr int TILE_BYTES = 128 * 256;  // [2 dim halves][128 rows][64] bf16, 128-byte swizzle
   static constexpr int OFF_Q = 0;
-  static constexpr int OFF_K = OFF_Q + 2 * Q_BYTES;
-  static constexpr int OFF_V = OFF_K + NS * KV_BYTES;
-  static constexpr int OFF_UNI = OFF_V + NS * KV_BYTES;  // int32[kMaxNb]: J | flags << 16
-  static constexpr int OFF_TBL = OFF_UNI + 4 * kMaxNb;   // uint32[kMaxNb]: flags per key block
-  static constexpr int OFF_BAR = OFF_TBL + 4 * kMaxNb;   // mbarriers and scalars
+  static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
+  static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
+  static constexpr int OFF_UNI = OFF_V + NS * TILE_BYTES;  // int32[kMaxNb]: J | flags << 16
+  static constexpr int OFF_TBL = OFF_UNI + 4 * kMaxNb;     // uint32[kMaxNb]: flags per key block
+  static constexpr int OFF_XCH = OFF_TBL + 4 * kMaxNb;     // float[2 tiles][2 halves][128 rows]: row max / sum exchange
+  static constexpr int OFF_BAR = OFF_XCH + 2048;           // mbarriers and scalars
   static constexpr int TOTAL = OFF_BAR + 512;
 };
 
 struct AttnBars {
   uint64_t q_full[2];
-  uint64_t k_full[4], k_empty[4], v_full[4], v_empty[4];
+  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
   uint64_t s_full[2], p_full[2], pv_done[2];
+  uint64_t x_full[2][4];  // [tile][lane quarter]: the two column halves of the same 32 rows meet here
   uint32_t tmem_base;
   int n_union;
   int abort;
@@ -67,17 +74,38 @@ struct AttnParams {
   float scale_log2;
 };
 
-template <int BK>
+#ifdef HEART_TRACE
+// Debug build only: clock64 stamps of CTA 0 written after the lse buffer (int64 [64 tiles][2][16] at lse + R*N).
+#define TRACE(k, t, slot)                                                                      \
+  do {                                                                                         \
+    if (blockIdx.x == 0 && (k) < 64 && p.lse != nullptr)                                       \
+      reinterpret_cast<long long *>(p.lse + (size_t)(gridDim.x / p.n_ctas_per_head) * p.N)[((k) * 2 + (t)) * 16 + (slot)] = clock64();          \
+  } while (0)
+#else
+#define TRACE(k, t, slot) \
+  do {                    \
+  } while (0)
+#endif
+
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+template <int B>
 __global__ void __launch_bounds__(kAttnThreads, 1)
     attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
                    const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
-  using L = AttnSmem<BK>;
+  using L = AttnSmem<B>;
+  constexpr int SUBS = L::SUBS;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) &
                                                           ~static_cast<uintptr_t>(1023));
   unsigned char *Qs = smem + L::OFF_Q, *Ks = smem + L::OFF_K, *Vs = smem + L::OFF_V;
   int32_t *uni = reinterpret_cast<int32_t *>(smem + L::OFF_UNI);
   uint32_t *tbl = reinterpret_cast<uint32_t *>(smem + L::OFF_TBL);
+  float *xch = reinterpret_cast<float *>(smem + L::OFF_XCH);
   AttnBars *bars = reinterpret_cast<AttnBars *>(smem + L::OFF_BAR);
   volatile int *abort = &bars->abort;
 
@@ -92,10 +120,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars->q_full[i], 1);
       mbar_init(&bars->s_full[i], 1);
-      mbar_init(&bars->p_full[i], 128);
+      mbar_init(&bars->p_full[i], 8);  // one arrival per softmax warp
+      for (int qq = 0; qq < 4; ++qq) mbar_init(&bars->x_full[i][qq], 2);
       mbar_init(&bars->pv_done[i], 1);
-    }
-    for (int i = 0; i < 4; ++i) {
       mbar_init(&bars->k_full[i], 1);
       mbar_init(&bars->k_empty[i], 1);
       mbar_init(&bars->v_full[i], 1);
@@ -153,33 +180,42 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
   const int U = bars->n_union;
+  const int NT = (U + SUBS - 1) / SUBS;  // 128-key tiles
   const uint32_t tile_mask0 = (1u << L::QBT) - 1u;
 
   // ------------------------------------------------------------------ roles
-  if (warp == 0) {
-    if (lane == 0) {  // ===== TMA producer
+  if (warp < 2) {
+    if (warp == 0 && lane == 0) {  // ===== TMA producer
       for (int t = 0; t < 2; ++t) {
         const int tr = row0 + t * 128;
         if (tr < p.N) {
-          mbar_expect_tx(&bars->q_full[t], L::Q_BYTES);
-          tma_load_4d(Qs + t * L::Q_BYTES, &map_q, &bars->q_full[t], 0, tr, hidx, bidx);
-          tma_load_4d(Qs + t * L::Q_BYTES + 128 * 128, &map_q, &bars->q_full[t], 64, tr, hidx, bidx);
+          mbar_expect_tx(&bars->q_full[t], L::TILE_BYTES);
+          tma_load_4d(Qs + t * L::TILE_BYTES, &map_q, &bars->q_full[t], 0, tr, hidx, bidx);
+          tma_load_4d(Qs + t * L::TILE_BYTES + 128 * 128, &map_q, &bars->q_full[t], 64, tr, hidx, bidx);
         }
       }
-      int n_k = 0, n_v = 0;  // K and V loads issued so far
-      for (int u = 0; u < U; ++u) {
-        const int s = u % L::NS, ph = (u / L::NS) & 1;
-        const int J = uni[u] & 0xffff;
-        if (u >= L::NS && !mbar_wait(&bars->k_empty[s], ph ^ 1, abort)) break;
-        mbar_expect_tx(&bars->k_full[s], L::KV_BYTES);
-        tma_load_4d(Ks + s * L::KV_BYTES, &map_kv, &bars->k_full[s], 0, J * BK, hidx, bidx);
-        tma_load_4d(Ks + s * L::KV_BYTES + BK * 128, &map_kv, &bars->k_full[s], 64, J * BK, hidx, bidx);
-        n_k = u + 1;
-        if (u >= L::NS && !mbar_wait(&bars->v_empty[s], ph ^ 1, abort)) break;
-        mbar_expect_tx(&bars->v_full[s], L::KV_BYTES);
-        tma_load_4d(Vs + s * L::KV_BYTES, &map_v, &bars->v_full[s], 0, J * BK, hidx, bidx);
-        tma_load_4d(Vs + s * L::KV_BYTES + BK * 128, &map_v, &bars->v_full[s], 64, J * BK, hidx, bidx);
-        n_v = u + 1;
+      int n_k = 0, n_v = 0;  // K and V tiles issued so far
+      for (int k = 0; k < NT; ++k) {
+        const int s = k & 1, ph = (k >> 1) & 1;
+        const int nsub = min(SUBS, U - k * SUBS);
+        if (k >= 2 && !mbar_wait(&bars->k_empty[s], ph ^ 1, abort)) break;
+        mbar_expect_tx(&bars->k_full[s], nsub * B * 256);
+        for (int sub = 0; sub < nsub; ++sub) {
+          const int J = uni[k * SUBS + sub] & 0xffff;
+          unsigned char *dst = Ks + s * L::TILE_BYTES + sub * (B * 128);
+          tma_load_4d(dst, &map_kv, &bars->k_full[s], 0, J * B, hidx, bidx);
+          tma_load_4d(dst + 128 * 128, &map_kv, &bars->k_full[s], 64, J * B, hidx, bidx);
+        }
+        n_k = k + 1;
+        if (k >= 2 && !mbar_wait(&bars->v_empty[s], ph ^ 1, abort)) break;
+        mbar_expect_tx(&bars->v_full[s], nsub * B * 256);
+        for (int sub = 0; sub < nsub; ++sub) {
+          const int J = uni[k * SUBS + sub] & 0xffff;
+          unsigned char *dst = Vs + s * L::TILE_BYTES + sub * (B * 128);
+          tma_load_4d(dst, &map_v, &bars->v_full[s], 0, J * B, hidx, bidx);
+          tma_load_4d(dst + 128 * 128, &map_v, &bars->v_full[s], 64, J * B, hidx, bidx);
+        }
+        n_v = k + 1;
       }
       // Shared memory must not be released under a copy in flight: the Q tiles are always awaited here
       // (nobody else does when the union is empty), and after an abort so are the last K/V copies.
@@ -191,39 +227,50 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       for (int t = 0; t < 2; ++t)
         if (row0 + t * 128 < p.N) settle(&bars->q_full[t], 0);
       if (*abort) {
-        for (int u = (n_k > L::NS ? n_k - L::NS : 0); u < n_k; ++u) settle(&bars->k_full[u % L::NS], (u / L::NS) & 1);
-        for (int u = (n_v > L::NS ? n_v - L::NS : 0); u < n_v; ++u) settle(&bars->v_full[u % L::NS], (u / L::NS) & 1);
+        for (int k = (n_k > 2 ? n_k - 2 : 0); k < n_k; ++k) settle(&bars->k_full[k & 1], (k >> 1) & 1);
+        for (int k = (n_v > 2 ? n_v - 2 : 0); k < n_v; ++k) settle(&bars->v_full[k & 1], (k >> 1) & 1);
       }
-    }
-  } else if (warp == 1) {
-    if (lane == 0 && U > 0) {  // ===== MMA issuer
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, BK, false, false);
+    } else if (warp == 1 && lane == 0 && NT > 0) {  // ===== MMA issuer
+      constexpr uint32_t idesc_qk_full = idesc_bf16_f32(128, 128, false, false);
+      constexpr uint32_t idesc_qk_half = idesc_bf16_f32(128, 64, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, 128, false, true);
       const uint32_t q_addr = smem_u32(Qs), k_addr = smem_u32(Ks), v_addr = smem_u32(Vs);
       uint32_t fresh_mask = 3u;  // bit t: O_t has not been written yet
       int n_pv0 = 0, n_pv1 = 0;
       bool ok = true;
-      auto active = [&](int u, int t) -> bool {
-        return (((uint32_t)uni[u] >> 16) & (tile_mask0 << (t * L::QBT))) != 0u;
-      };
-      auto issue_qk = [&](int t, int u) {
-        const int s = u % L::NS;
+      auto keys_in = [&](int k) -> int { return min(SUBS, U - k * SUBS) * B; };
+      auto active = [&](int k, int t) -> bool {
+        uint32_t f = 0;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t a = smem_desc_sw128(q_addr + t * L::Q_BYTES + (ks >> 2) * (128 * 128) + (ks & 3) * 32, 16, 1024);
-          const uint64_t b = smem_desc_sw128(k_addr + s * L::KV_BYTES + (ks >> 2) * (BK * 128) + (ks & 3) * 32, 16, 1024);
-          mma_ss(tmem + t * 128, a, b, idesc_qk, ks > 0 ? 1u : 0u);
-        }
+        for (int sub = 0; sub < SUBS; ++sub)
+          if (k * SUBS + sub < U) f |= (uint32_t)uni[k * SUBS + sub] >> 16;
+        return (f & (tile_mask0 << (t * L::QBT))) != 0u;
+      };
+      // descriptors differ only in the 14-bit start-address field: base + constant per k-step
+      const uint64_t q_desc = smem_desc_sw128(q_addr, 16, 1024);
+      const uint64_t k_desc = smem_desc_sw128(k_addr, 16, 1024);
+      const uint64_t v_desc = smem_desc_sw128(v_addr, 128 * 128, 1024);
+      auto issue_qk = [&](int t, int k) {
+        const uint64_t a0 = q_desc + (uint64_t)(t * (L::TILE_BYTES >> 4));
+        const uint64_t b0 = k_desc + (uint64_t)((k & 1) * (L::TILE_BYTES >> 4));
+        const uint32_t d = tmem + t * 128;
+        const uint32_t idesc = keys_in(k) == 128 ? idesc_qk_full : idesc_qk_half;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          mma_ss(d, a0 + ((ks >> 2) * 1024 + (ks & 3) * 2), b0 + ((ks >> 2) * 1024 + (ks & 3) * 2), idesc, ks > 0 ? 1u : 0u);
         tc_commit(&bars->s_full[t]);
       };
-      auto issue_pv = [&](int t, int u) {
-        const int s = u % L::NS;
-#pragma unroll
-        for (int ks = 0; ks < BK / 16; ++ks) {
-          const uint64_t b = smem_desc_sw128(v_addr + s * L::KV_BYTES + ks * 2048, BK * 128, 1024);
-          mma_ts(tmem + 256 + t * 128, tmem + t * 128 + ks * 8, b, idesc_pv, (((fresh_mask >> t) & 1u) && ks == 0) ? 0u : 1u);
-        }
+      auto issue_pv = [&](int t, int k) {
+        const uint64_t b0 = v_desc + (uint64_t)((k & 1) * (L::TILE_BYTES >> 4));
+        const uint32_t d = tmem + 256 + t * 128, pa = tmem + t * 128;
+        mma_ts(d, pa, b0, idesc_pv, ((fresh_mask >> t) & 1u) ? 0u : 1u);
         fresh_mask &= ~(1u << t);
+#pragma unroll
+        for (int ks = 1; ks < 4; ++ks) mma_ts(d, pa + ks * 8, b0 + ks * 128, idesc_pv, 1u);
+        if (keys_in(k) == 128) {
+#pragma unroll
+          for (int ks = 4; ks < 8; ++ks) mma_ts(d, pa + ks * 8, b0 + ks * 128, idesc_pv, 1u);
+        }
         tc_commit(&bars->pv_done[t]);
       };
       for (int t = 0; t < 2 && ok; ++t)
@@ -235,65 +282,100 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         if (active(0, 1)) issue_qk(1, 0);
         tc_commit(&bars->k_empty[0]);
       }
-      for (int u = 0; u < U && ok; ++u) {
-        const int s = u % L::NS, ph = (u / L::NS) & 1;
-        const bool more = (u + 1 < U);
+      for (int k = 0; k < NT && ok; ++k) {
+        const int s = k & 1, ph = (k >> 1) & 1;
+        const bool more = (k + 1 < NT);
         ok = mbar_wait(&bars->v_full[s], ph, abort);
-        if (ok && more) ok = mbar_wait(&bars->k_full[(u + 1) % L::NS], ((u + 1) / L::NS) & 1, abort);
+        if (ok && more) ok = mbar_wait(&bars->k_full[(k + 1) & 1], ((k + 1) >> 1) & 1, abort);
         if (!ok) break;
         tc_fence_after();
         for (int t = 0; t < 2 && ok; ++t) {
-          if (active(u, t)) {
+          if (active(k, t)) {
             int &n_pv = t ? n_pv1 : n_pv0;
             ok = mbar_wait(&bars->p_full[t], n_pv & 1, abort);
             if (!ok) break;
             ++n_pv;
             tc_fence_after();
-            issue_pv(t, u);
+            issue_pv(t, k);
           }
-          if (more && active(u + 1, t)) issue_qk(t, u + 1);
+          if (more && active(k + 1, t)) issue_qk(t, k + 1);
         }
         if (!ok) break;
         tc_commit(&bars->v_empty[s]);
-        if (more) tc_commit(&bars->k_empty[(u + 1) % L::NS]);
+        if (more) tc_commit(&bars->k_empty[(k + 1) & 1]);
       }
     }
-  } else if (warp >= 4) {
-    // ===== softmax / correction / epilogue: warpgroup t handles tile t, thread = query row
-    const int t = (warp - 4) >> 2;
-    const int q = warp & 3;                 // TMEM lane quarter this warp may touch
-    const int row_in_tile = q * 32 + lane;
-    const int tok = row0 + t * 128 + row_in_tile;
-    const bool valid_row = tok < p.N;
-    const uint32_t my_bit = 1u << (t * L::QBT + row_in_tile / BK);
-    const uint32_t my_tile_mask = tile_mask0 << (t * L::QBT);
-    const uint32_t s_addr = tmem + ((uint32_t)(q * 32) << 16) + t * 128;
-    const uint32_t o_addr = tmem + ((uint32_t)(q * 32) << 16) + 256 + t * 128;
+  } else {
+    // ===== softmax / correction / epilogue: thread = (query row of either tile, half of the key columns)
+    // The tile index t is a run-time value on purpose: one compact copy of this code serves both
+    // tiles, which keeps the loop inside the instruction cache.
+    const int a = (warp - 2) >> 2;  // column half: S columns [64a, 64a+64), O columns [64a, 64a+64)
+    const int q = warp & 3;         // TMEM lane quarter this warp may touch
+    const int row = q * 32 + lane;  // row inside a 128-row query tile
+    const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const float c = p.scale_log2;
-    float m_ref = -INFINITY, l = 0.f;
-    int n_act = 0;
+    float m_ref0 = -INFINITY, m_ref1 = -INFINITY, l_part0 = 0.f, l_part1 = 0.f;
+    int n_act0 = 0, n_act1 = 0;
     bool ok = true;
-    for (int u = 0; u < U && ok; ++u) {
-      const uint32_t e = (uint32_t)uni[u];
-      if (((e >> 16) & my_tile_mask) == 0u) continue;
-      const int J = e & 0xffff;
-      const bool row_has = ((e >> 16) & my_bit) != 0u;
-      const int kv_valid = row_has ? min(BK, p.N - J * BK) : 0;
+    const int my_sub = (a * 64) / B;           // key sub-block this thread's columns belong to
+    const int col_in_sub = a * 64 - my_sub * B;  // first of its columns inside that sub-block
+    for (int kt = 0; kt < 2 * NT && ok; ++kt) {
+      const int k = kt >> 1, t = kt & 1;
+      const int nsub = min(SUBS, U - k * SUBS);
+      // valid key columns, for this row, of the thread's two 32-column chunks
+      uint32_t tile_flags = 0;
+      int lim0 = 0, lim1 = 0;
+      {
+        const uint32_t my_bit = 1u << (t * L::QBT + row / B);  // uniform within a warp
+#pragma unroll
+        for (int sub = 0; sub < SUBS; ++sub) {
+          if (sub < nsub) {
+            const uint32_t e = (uint32_t)uni[k * SUBS + sub];
+            tile_flags |= e >> 16;
+            if (sub == my_sub && ((e >> 16) & my_bit)) {
+              const int v = min(B, p.N - (int)(e & 0xffff) * B) - col_in_sub;
+              lim0 = max(0, min(32, v));
+              lim1 = max(0, min(32, v - 32));
+            }
+          }
+        }
+      }
+      if ((tile_flags & (tile_mask0 << (t * L::QBT))) == 0u) continue;
+      const int n_act = t ? n_act1 : n_act0;
+      float m_ref = t ? m_ref1 : m_ref0;
+      const uint32_t s_addr = lane_addr + t * 128 + a * 64;
+      const uint32_t o_addr = lane_addr + 256 + t * 128 + a * 64;
+      float *xrow = xch + (t * 2) * 128 + row;  // [t][half][row]
       ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[t], n_act & 1, abort));
       if (!ok) break;
       tc_fence_after();
-      // pass 1: row maximum of the raw scores
-      float mx = -INFINITY;
+      uint32_t sreg[64];
+      if (lim0 > 0) tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
+      if (lim1 > 0) tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
+      tmem_wait_ld();
+      if (lim0 < 32 || lim1 < 32) {  // rare: ragged last block or a sub-block this row does not list
 #pragma unroll
-      for (int ch = 0; ch < BK / 32; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(s_addr + ch * 32, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (ch * 32 + i < kv_valid) mx = fmaxf(mx, __uint_as_float(v[i]));
+        for (int i = 0; i < 32; ++i) {
+          if (i >= lim0) sreg[i] = 0xff800000u;  // -inf: ignored by the max, 2^-inf = 0
+          if (i >= lim1) sreg[32 + i] = 0xff800000u;
+        }
       }
-      const float x_max = mx * c;  // -inf stays -inf (c > 0)
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 64; i += 8) {
+        mx0 = fmax3(mx0, __uint_as_float(sreg[i]), __uint_as_float(sreg[i + 1]));
+        mx1 = fmax3(mx1, __uint_as_float(sreg[i + 2]), __uint_as_float(sreg[i + 3]));
+        mx2 = fmax3(mx2, __uint_as_float(sreg[i + 4]), __uint_as_float(sreg[i + 5]));
+        mx3 = fmax3(mx3, __uint_as_float(sreg[i + 6]), __uint_as_float(sreg[i + 7]));
+      }
+      // the two column halves of a row exchange their maxima
+      const float mx_mine = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      xrow[a * 128] = mx_mine;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->x_full[t][q]);
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[t][q], n_act & 1, abort));
+      if (!ok) break;
+      const float x_max = fmaxf(mx_mine, xrow[(1 - a) * 128]) * c;  // -inf stays -inf (c > 0)
       float alpha = 1.f;
       bool grow = false;
       if (m_ref == -INFINITY) {
@@ -308,8 +390,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[t], (n_act - 1) & 1, abort));
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
+#pragma unroll 1
+        for (int ch = 0; ch < 2; ++ch) {
           uint32_t v[32];
           tmem_ld32(o_addr + ch * 32, v);
           tmem_wait_ld();
@@ -319,41 +401,70 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         tmem_wait_st();
       }
-      l *= alpha;
-      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-      // pass 2: p = 2^(s*c - m), packed to bf16 over the first BK/2 columns of S_t
-      float sum = 0.f;
+      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      // p = 2^(s*c - m), packed to bf16 over columns [32a, 32a+32) of S_t
+      float sum0 = 0.f, sum1 = 0.f;
+      if (a * 64 < nsub * B) {  // else: sub-block absent from this tile, the PV product skips its keys
 #pragma unroll
-      for (int ch = 0; ch < BK / 32; ++ch) {
-        uint32_t v[32], pk[16];
-        tmem_ld32(s_addr + ch * 32, v);
-        tmem_wait_ld();
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t pk[16];
+          if ((ch ? lim1 : lim0) == 0) {  // this row lists nothing here: zeros, no exponentials
 #pragma unroll
-        for (int i = 0; i < 32; i += 2) {
-          const float p0 = (ch * 32 + i < kv_valid) ? ex2(fmaf(__uint_as_float(v[i]), c, -m_use)) : 0.f;
-          const float p1 = (ch * 32 + i + 1 < kv_valid) ? ex2(fmaf(__uint_as_float(v[i + 1]), c, -m_use)) : 0.f;
-          // the row sum is taken over the bf16-rounded weights, the ones the PV product really uses,
-          // so numerator and denominator carry the same rounding and O stays a true weighted mean
-          const uint32_t w = pack_bf16x2(p0, p1);
-          pk[i >> 1] = w;
-          sum += __uint_as_float(w << 16) + __uint_as_float(w & 0xffff0000u);
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+          } else
+#pragma unroll
+          for (int i = 0; i < 32; i += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(sreg[ch * 32 + i]), c, neg_m));
+            const float p1 = ex2(fmaf(__uint_as_float(sreg[ch * 32 + i + 1]), c, neg_m));
+            // the row sum is taken over the bf16-rounded weights, the ones the PV product really
+            // uses, so numerator and denominator carry the same rounding: O stays a weighted mean
+            const uint32_t w = pack_bf16x2(p0, p1);
+            pk[i >> 1] = w;
+            sum0 += __uint_as_float(w << 16);
+            sum1 += __uint_as_float(w & 0xffff0000u);
+          }
+          tmem_st16(lane_addr + t * 128 + a * 32 + ch * 16, pk);
         }
-        tmem_st16(s_addr + ch * 16, pk);
       }
-      l += sum;
+      const float l_new = (t ? l_part1 : l_part0) * alpha + (sum0 + sum1);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bars->p_full[t]);
-      ++n_act;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->p_full[t]);
+      if (t) {
+        m_ref1 = m_ref;
+        l_part1 = l_new;
+        ++n_act1;
+      } else {
+        m_ref0 = m_ref;
+        l_part0 = l_new;
+        ++n_act0;
+      }
     }
-    // epilogue
-    if (ok && n_act > 0) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[t], (n_act - 1) & 1, abort));
-    if (ok) {
+    // epilogue: each warpgroup writes its 64-dim half of both tiles' output rows
+#pragma unroll 1
+    for (int t = 0; t < 2; ++t) {
+      const int tok = row0 + t * 128 + row;
+      const bool valid_row = tok < p.N;
+      const int n_act = t ? n_act1 : n_act0;
+      const float m_ref = t ? m_ref1 : m_ref0;
+      const uint32_t o_addr = lane_addr + 256 + t * 128 + a * 64;
+      float *xrow = xch + (t * 2) * 128 + row;
+      float l = t ? l_part1 : l_part0;
+      if (ok && n_act > 0) {
+        xrow[a * 128] = l;  // the halves add their partial row sums
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->x_full[t][q]);
+        ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[t][q], n_act & 1, abort));
+        if (ok) l += xrow[(1 - a) * 128];
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[t], (n_act - 1) & 1, abort));
+      }
+      if (!ok) break;
       tc_fence_after();
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      uint16_t *orow = p.O + (long long)bidx * p.sb + (long long)hidx * p.sh + (long long)tok * p.sn;
-#pragma unroll
-      for (int ch = 0; ch < 4; ++ch) {
+      uint16_t *orow = p.O + (long long)bidx * p.sb + (long long)hidx * p.sh + (long long)tok * p.sn + a * 64;
+#pragma unroll 1
+      for (int ch = 0; ch < 2; ++ch) {
         uint32_t v[32];
         if (n_act > 0) {
           tmem_ld32(o_addr + ch * 32, v);
@@ -374,7 +485,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
         }
       }
-      if (valid_row && p.lse != nullptr)
+      if (a == 0 && valid_row && p.lse != nullptr)
         p.lse[(size_t)r * p.N + tok] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
@@ -422,13 +533,13 @@ bool make_map(CUtensorMap *m, const void *base, const Geom &g, int rows) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BK>
+template <int B>
 cudaError_t launch_bk(const Geom &g, const CUtensorMap &mq, const CUtensorMap &mk, const CUtensorMap &mv,
                       const AttnParams &prm, cudaStream_t s) {
-  const int smem = AttnSmem<BK>::TOTAL + 1024;
-  cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const int smem = AttnSmem<B>::TOTAL + 1024;
+  cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  attn_tc_kernel<BK><<<g.R * prm.n_ctas_per_head, kAttnThreads, smem, s>>>(mq, mk, mv, prm);
+  attn_tc_kernel<B><<<g.R * prm.n_ctas_per_head, kAttnThreads, smem, s>>>(mq, mk, mv, prm);
   return cudaGetLastError();
 }
 

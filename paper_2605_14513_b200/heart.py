@@ -12,7 +12,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libheart.so")
+_LIB_PATH = os.environ.get("HEART_LIB") or os.path.join(_HERE, "libheart.so")
 
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
 STATIC_SCRATCH_BYTES = 16 << 20
