@@ -94,7 +94,8 @@ class ClockSampler:
 
 
 def retained_flops(torch, st, wl):
-    """4 * (real query rows) * (real key rows) * D summed over the retained pairs (never padding)."""
+    """4 * (real query rows) * (real key rows) * D summed over the retained pairs (never padding).
+    Returns device scalars (flops, pairs): no host synchronisation."""
     nb, b, N = wl.n_blocks, wl.block, wl.N
     last = N - (nb - 1) * b
     cnt = st.kv_cnt.to(torch.float64)                                    # [R, nb]
@@ -102,7 +103,7 @@ def retained_flops(torch, st, wl):
     keys = cnt * b - has_last * (b - last)                               # real key rows per query block
     qrows = torch.full((nb,), float(b), dtype=torch.float64, device=cnt.device)
     qrows[nb - 1] = last
-    return float(4.0 * wl.D * (keys * qrows[None, :]).sum().item()), float(cnt.sum().item())
+    return 4.0 * wl.D * (keys * qrows[None, :]).sum(), cnt.sum()
 
 
 def run_ours(args, rank, world):
@@ -176,10 +177,11 @@ def run_ours(args, rank, world):
         total_ms = float(tt.item())
     ms_per_step = total_ms / K
 
-    # ---- per-stage pass: the same K steps as three C-ABI calls, one event pair per call
+    # ---- per-stage pass: the same K steps as three C-ABI calls, one event pair per call.  Nothing here
+    # synchronises with the host: the flop / pair / refresh counts are accumulated on the device.
     st.load_state_dict(ckpt)
     stage_ev = []
-    flops_total = pairs_total = refreshed = 0.0
+    acc = torch.zeros(3, dtype=torch.float64, device=dev)  # retained flops, retained pairs, refreshed heads
     r2 = torch.empty_like(refresh)
     for k in range(K):
         Q, Kt, V = steps_in[W + k]
@@ -192,11 +194,10 @@ def run_ours(args, rank, world):
         heart.heart_block_sparse_attn(cfg, Q, Kt, V, st.kv_idx, st.kv_cnt, O, ws)
         e[3].record()
         stage_ev.append(e)
-        torch.cuda.synchronize()
         f, p = retained_flops(torch, st, wl)
-        flops_total += f
-        pairs_total += p
-        refreshed += float(r2.sum().item())
+        acc += torch.stack([f, p, r2.sum().to(torch.float64)])
+    torch.cuda.synchronize()
+    flops_total, pairs_total, refreshed = (float(x) for x in acc.tolist())
     ms_drift = sum(e[0].elapsed_time(e[1]) for e in stage_ev) / K
     ms_mask = sum(e[1].elapsed_time(e[2]) for e in stage_ev) / K
     ms_attn = sum(e[2].elapsed_time(e[3]) for e in stage_ev) / K
@@ -239,8 +240,10 @@ def run_ours(args, rank, world):
     out = None
     if rank == 0:
         peak_tf = pk["bf16_tflops_sustained"]
+        # DRAM bytes per attention launch from the ncu capture summarised in profiles/ (this workload only)
+        traffic = {"wan1.3b-480p": 385.2e6}.get(wl.name)
         roofline = {"kernel": "block-sparse attention", "bound": "tensor", "achieved": attn_tflops, "peak": peak_tf,
-                    "unit": "TFLOP/s", "frac": attn_tflops / peak_tf, "traffic": None,
+                    "unit": "TFLOP/s", "frac": attn_tflops / peak_tf, "traffic": traffic,
                     "peak_source": pk["source"] + " (sustained bf16 cuBLAS, kernel timed inside a long step)",
                     "flops_per_launch": flops_step, "ms_per_launch": ms_attn}
         hbm = stats_bytes / (ms_drift * 1e-3) / 1e9

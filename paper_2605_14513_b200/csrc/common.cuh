@@ -20,8 +20,11 @@ struct Geom {
 
 // Chunking of the block-sum pass: about 8 CTAs per SM on a 148-SM part, whatever the device (the
 // split fixes the summation order, so it must depend on the shape only).
+#ifndef HEART_CHUNK_TARGET
+#define HEART_CHUNK_TARGET (148 * 8)
+#endif
 __host__ inline void set_chunks(Geom &g) {
-  const int target = 148 * 8;
+  const int target = HEART_CHUNK_TARGET;
   int per_pair = (target + 2 * g.R - 1) / (2 * g.R);
   if (per_pair < 1) per_pair = 1;
   g.bpc = (g.nb + per_pair - 1) / per_pair;
