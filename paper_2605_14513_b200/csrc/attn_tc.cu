@@ -1,25 +1,25 @@
 // Block-sparse attention with online softmax on the sm_100a tensor cores.
 //
-// One CTA owns 256 consecutive query rows of one head = two 128-row MMA tiles (tile t = rows
-// [128t, 128t+128)).  With 128-token blocks a tile is one query block; with 64-token blocks it is two
-// query blocks whose lists are merged (rows of the half that does not list a key block see -inf).
-// The lists of the CTA's 2 or 4 query blocks are merged once into an ascending union; each union
-// entry carries one flag bit per query block.  K/V blocks are fetched once per CTA and shared by
-// both tiles; a tile skips the MMAs of union entries none of its query blocks lists.
+// One CTA owns one 128-row query tile of one head: one query block of 128 tokens, or two query
+// blocks of 64 whose lists are merged into an ascending union (one flag bit per query block; rows of
+// the half that does not list a key block see -inf there).  Keys are processed 128 at a time: a key
+// tile is one 128-token block or two 64-token blocks of the union.
+//
+// The key tiles are dealt to two independent streams (even / odd tile index).  Each stream keeps its
+// own running max, row sum and output accumulator and the two are merged at the end, so the softmax of
+// one stream overlaps the MMAs of the other (ping-pong) although both work for the same query rows.
 //
 // Warp roles (320 threads):
-//   warp 0      TMA producer: Q tiles once, then the listed K and V blocks through shared-memory
+//   warp 0      TMA producer: the Q tile once, then the listed K and V blocks through shared-memory
 //               rings (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers).
-//   warp 1      MMA issuer (one lane): S_t = Q_t K^T into tensor memory (tcgen05.mma, operands in
-//               shared memory), O_t += P_t V with P_t read from tensor memory; the two tiles are
-//               interleaved so one tile's softmax overlaps the other tile's MMAs.
-//   warps 2-9   softmax: both warpgroups work on the tile whose scores are ready, warpgroup a on key
+//   warp 1      MMA issuer (one lane): S_t = Q K^T into tensor memory (tcgen05.mma, operands in shared
+//               memory), O_t += P_t V with P_t read from tensor memory.
+//   warps 2-9   softmax: both warpgroups work on the stream whose scores are ready, warpgroup a on key
 //               columns [64a, 64a+64); thread = (query row, column half).  It reads its half of the S
 //               row from tensor memory, the two halves exchange their row maxima through shared
 //               memory, it keeps the running max / partial sum, writes P (bf16) back over S,
-//               rescales its half of O only when the max grew by more than 2^8, and writes its half
-//               of O (and lse) at the end.  Two warps per scheduler work at the same time, so the
-//               exponentials (MUFU) of one overlap the FMA/ALU work of the other.
+//               rescales its half of O only when the max grew by more than 2^8, and at the end merges
+//               the two streams and writes its half of O (and lse).
 // Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P_t aliases S_t.
 //
 // Every wait is bounded; a wait that runs out raises a CTA-wide abort flag and the status word, the
@@ -38,26 +38,24 @@ constexpr int kMaxNb = HEART_MAX_BLOCKS;
 // Shared-memory plan.  A key tile always holds 128 keys = SUBS key blocks of B tokens.
 template <int B>
 struct AttnSmem {
-  static constexpr int SUBS = 128 / B;       // key blocks per 128-key tile (1 or 2)
-  static constexpr int NQB = 256 / B;        // query blocks per CTA (2 or 4)
-  static constexpr int QBT = 128 / B;        // query blocks per 128-row query tile
-  static constexpr int NS = 2;               // ring depth of K and of V
+  static constexpr int SUBS = 128 / B;          // key blocks per 128-key tile (1 or 2)
+  static constexpr int QBT = 128 / B;           // query blocks per CTA (1 or 2)
   static constexpr int TILE_BYTES = 128 * 256;  // [2 dim halves][128 rows][64] bf16, 128-byte swizzle
   static constexpr int OFF_Q = 0;
-  static constexpr int OFF_K = OFF_Q + 2 * TILE_BYTES;
-  static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
-  static constexpr int OFF_UNI = OFF_V + NS * TILE_BYTES;  // int32[kMaxNb]: J | flags << 16
-  static constexpr int OFF_TBL = OFF_UNI + 4 * kMaxNb;     // uint32[kMaxNb]: flags per key block
-  static constexpr int OFF_XCH = OFF_TBL + 4 * kMaxNb;     // float[2 tiles][2 halves][128 rows]: row max / sum exchange
-  static constexpr int OFF_BAR = OFF_XCH + 2048;           // mbarriers and scalars
+  static constexpr int OFF_K = OFF_Q + TILE_BYTES;      // 2 stages: stream t uses stage t
+  static constexpr int OFF_V = OFF_K + 2 * TILE_BYTES;  // 2 stages
+  static constexpr int OFF_UNI = OFF_V + 2 * TILE_BYTES;  // int32[kMaxNb]: J | flags << 16
+  static constexpr int OFF_TBL = OFF_UNI + 4 * kMaxNb;    // uint32[kMaxNb]: flags per key block
+  static constexpr int OFF_XCH = OFF_TBL + 4 * kMaxNb;    // float[2 uses][2 streams][2 halves][128 rows]: row max, row sum
+  static constexpr int OFF_BAR = OFF_XCH + 4096;          // mbarriers and scalars
   static constexpr int TOTAL = OFF_BAR + 512;
 };
 
 struct AttnBars {
-  uint64_t q_full[2];
+  uint64_t q_full;
   uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
   uint64_t s_full[2], p_full[2], pv_done[2];
-  uint64_t x_full[2][4];  // [tile][lane quarter]: the two column halves of the same 32 rows meet here
+  uint64_t x_full[2][4];  // [stream][lane quarter]: the two column halves of the same 32 rows meet here
   uint32_t tmem_base;
   int n_union;
   int abort;
@@ -73,19 +71,6 @@ struct AttnParams {
   int H, N, nb, idx_stride, n_ctas_per_head, dense;
   float scale_log2;
 };
-
-#ifdef HEART_TRACE
-// Debug build only: clock64 stamps of CTA 0 written after the lse buffer (int64 [64 tiles][2][16] at lse + R*N).
-#define TRACE(k, t, slot)                                                                      \
-  do {                                                                                         \
-    if (blockIdx.x == 0 && (k) < 64 && p.lse != nullptr)                                       \
-      reinterpret_cast<long long *>(p.lse + (size_t)(gridDim.x / p.n_ctas_per_head) * p.N)[((k) * 2 + (t)) * 16 + (slot)] = clock64();          \
-  } while (0)
-#else
-#define TRACE(k, t, slot) \
-  do {                    \
-  } while (0)
-#endif
 
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float r;
@@ -112,13 +97,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int r = blockIdx.x / p.n_ctas_per_head, cta_in_head = blockIdx.x % p.n_ctas_per_head;
   const int bidx = r / p.H, hidx = r % p.H;
-  const int row0 = cta_in_head * 256;  // first query token of this CTA
+  const int row0 = cta_in_head * 128;  // first query token of this CTA
   const int nb = p.nb;
 
   // ------------------------------------------------------------------ set-up
   if (tid == 0) {
+    mbar_init(&bars->q_full, 1);
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&bars->q_full[i], 1);
       mbar_init(&bars->s_full[i], 1);
       mbar_init(&bars->p_full[i], 8);  // one arrival per softmax warp
       for (int qq = 0; qq < 4; ++qq) mbar_init(&bars->x_full[i][qq], 2);
@@ -135,8 +120,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   }
   for (int j = tid; j < nb; j += kAttnThreads) tbl[j] = 0u;
   __syncthreads();
-  for (int qb = 0; qb < L::NQB; ++qb) {  // scatter: flag bit qb of every key block listed by query block qb
-    const int I = cta_in_head * L::NQB + qb;
+  for (int qb = 0; qb < L::QBT; ++qb) {  // scatter: flag bit qb of every key block listed by query block qb
+    const int I = cta_in_head * L::QBT + qb;
     if (I >= nb) break;
     const size_t row = (size_t)r * nb + I;
     int cnt = p.dense ? nb : p.kv_cnt[row];
@@ -180,20 +165,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
   const int U = bars->n_union;
-  const int NT = (U + SUBS - 1) / SUBS;  // 128-key tiles
-  const uint32_t tile_mask0 = (1u << L::QBT) - 1u;
+  const int NT = (U + SUBS - 1) / SUBS;  // 128-key tiles; tile k belongs to stream k & 1
 
   // ------------------------------------------------------------------ roles
   if (warp < 2) {
     if (warp == 0 && lane == 0) {  // ===== TMA producer
-      for (int t = 0; t < 2; ++t) {
-        const int tr = row0 + t * 128;
-        if (tr < p.N) {
-          mbar_expect_tx(&bars->q_full[t], L::TILE_BYTES);
-          tma_load_4d(Qs + t * L::TILE_BYTES, &map_q, &bars->q_full[t], 0, tr, hidx, bidx);
-          tma_load_4d(Qs + t * L::TILE_BYTES + 128 * 128, &map_q, &bars->q_full[t], 64, tr, hidx, bidx);
-        }
-      }
+      mbar_expect_tx(&bars->q_full, L::TILE_BYTES);
+      tma_load_4d(Qs, &map_q, &bars->q_full, 0, row0, hidx, bidx);
+      tma_load_4d(Qs + 128 * 128, &map_q, &bars->q_full, 64, row0, hidx, bidx);
       int n_k = 0, n_v = 0;  // K and V tiles issued so far
       for (int k = 0; k < NT; ++k) {
         const int s = k & 1, ph = (k >> 1) & 1;
@@ -217,15 +196,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         n_v = k + 1;
       }
-      // Shared memory must not be released under a copy in flight: the Q tiles are always awaited here
+      // Shared memory must not be released under a copy in flight: the Q tile is always awaited here
       // (nobody else does when the union is empty), and after an abort so are the last K/V copies.
       auto settle = [&](uint64_t *bar, uint32_t parity) {
         const long long t0 = clock64();
         while (!mbar_try_wait(bar, parity) && clock64() - t0 < 40000000LL) {
         }
       };
-      for (int t = 0; t < 2; ++t)
-        if (row0 + t * 128 < p.N) settle(&bars->q_full[t], 0);
+      settle(&bars->q_full, 0);
       if (*abort) {
         for (int k = (n_k > 2 ? n_k - 2 : 0); k < n_k; ++k) settle(&bars->k_full[k & 1], (k >> 1) & 1);
         for (int k = (n_v > 2 ? n_v - 2 : 0); k < n_v; ++k) settle(&bars->v_full[k & 1], (k >> 1) & 1);
@@ -234,37 +212,28 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       constexpr uint32_t idesc_qk_full = idesc_bf16_f32(128, 128, false, false);
       constexpr uint32_t idesc_qk_half = idesc_bf16_f32(128, 64, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, 128, false, true);
-      const uint32_t q_addr = smem_u32(Qs), k_addr = smem_u32(Ks), v_addr = smem_u32(Vs);
-      uint32_t fresh_mask = 3u;  // bit t: O_t has not been written yet
-      int n_pv0 = 0, n_pv1 = 0;
+      // descriptors differ only in the 14-bit start-address field: base + constant per k-step
+      const uint64_t q_desc = smem_desc_sw128(smem_u32(Qs), 16, 1024);
+      const uint64_t k_desc = smem_desc_sw128(smem_u32(Ks), 16, 1024);
+      const uint64_t v_desc = smem_desc_sw128(smem_u32(Vs), 128 * 128, 1024);
       bool ok = true;
       auto keys_in = [&](int k) -> int { return min(SUBS, U - k * SUBS) * B; };
-      auto active = [&](int k, int t) -> bool {
-        uint32_t f = 0;
-#pragma unroll
-        for (int sub = 0; sub < SUBS; ++sub)
-          if (k * SUBS + sub < U) f |= (uint32_t)uni[k * SUBS + sub] >> 16;
-        return (f & (tile_mask0 << (t * L::QBT))) != 0u;
-      };
-      // descriptors differ only in the 14-bit start-address field: base + constant per k-step
-      const uint64_t q_desc = smem_desc_sw128(q_addr, 16, 1024);
-      const uint64_t k_desc = smem_desc_sw128(k_addr, 16, 1024);
-      const uint64_t v_desc = smem_desc_sw128(v_addr, 128 * 128, 1024);
-      auto issue_qk = [&](int t, int k) {
-        const uint64_t a0 = q_desc + (uint64_t)(t * (L::TILE_BYTES >> 4));
-        const uint64_t b0 = k_desc + (uint64_t)((k & 1) * (L::TILE_BYTES >> 4));
+      auto issue_qk = [&](int k) {  // S_t = Q K_k^T, t = k & 1; K_k sits in stage t
+        const int t = k & 1;
+        const uint64_t b0 = k_desc + (uint64_t)(t * (L::TILE_BYTES >> 4));
         const uint32_t d = tmem + t * 128;
         const uint32_t idesc = keys_in(k) == 128 ? idesc_qk_full : idesc_qk_half;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          mma_ss(d, a0 + ((ks >> 2) * 1024 + (ks & 3) * 2), b0 + ((ks >> 2) * 1024 + (ks & 3) * 2), idesc, ks > 0 ? 1u : 0u);
+          mma_ss(d, q_desc + ((ks >> 2) * 1024 + (ks & 3) * 2), b0 + ((ks >> 2) * 1024 + (ks & 3) * 2), idesc, ks > 0 ? 1u : 0u);
         tc_commit(&bars->s_full[t]);
+        tc_commit(&bars->k_empty[t]);
       };
-      auto issue_pv = [&](int t, int k) {
-        const uint64_t b0 = v_desc + (uint64_t)((k & 1) * (L::TILE_BYTES >> 4));
+      auto issue_pv = [&](int k) {  // O_t (+)= P_t V_k
+        const int t = k & 1;
+        const uint64_t b0 = v_desc + (uint64_t)(t * (L::TILE_BYTES >> 4));
         const uint32_t d = tmem + 256 + t * 128, pa = tmem + t * 128;
-        mma_ts(d, pa, b0, idesc_pv, ((fresh_mask >> t) & 1u) ? 0u : 1u);
-        fresh_mask &= ~(1u << t);
+        mma_ts(d, pa, b0, idesc_pv, k >= 2 ? 1u : 0u);
 #pragma unroll
         for (int ks = 1; ks < 4; ++ks) mma_ts(d, pa + ks * 8, b0 + ks * 128, idesc_pv, 1u);
         if (keys_in(k) == 128) {
@@ -272,76 +241,58 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           for (int ks = 4; ks < 8; ++ks) mma_ts(d, pa + ks * 8, b0 + ks * 128, idesc_pv, 1u);
         }
         tc_commit(&bars->pv_done[t]);
+        tc_commit(&bars->v_empty[t]);
       };
-      for (int t = 0; t < 2 && ok; ++t)
-        if (row0 + t * 128 < p.N) ok = mbar_wait(&bars->q_full[t], 0, abort);
-      if (ok) ok = mbar_wait(&bars->k_full[0], 0, abort);
-      if (ok) {
-        tc_fence_after();
-        if (active(0, 0)) issue_qk(0, 0);
-        if (active(0, 1)) issue_qk(1, 0);
-        tc_commit(&bars->k_empty[0]);
+      ok = mbar_wait(&bars->q_full, 0, abort);
+      for (int k = 0; k < 2 && k < NT && ok; ++k) {
+        ok = mbar_wait(&bars->k_full[k], 0, abort);
+        if (ok) {
+          tc_fence_after();
+          issue_qk(k);
+        }
       }
       for (int k = 0; k < NT && ok; ++k) {
-        const int s = k & 1, ph = (k >> 1) & 1;
-        const bool more = (k + 1 < NT);
-        ok = mbar_wait(&bars->v_full[s], ph, abort);
-        if (ok && more) ok = mbar_wait(&bars->k_full[(k + 1) & 1], ((k + 1) >> 1) & 1, abort);
+        const int t = k & 1, ph = (k >> 1) & 1;
+        ok = mbar_wait(&bars->v_full[t], ph, abort);
+        if (ok) ok = mbar_wait(&bars->p_full[t], ph, abort);
         if (!ok) break;
         tc_fence_after();
-        for (int t = 0; t < 2 && ok; ++t) {
-          if (active(k, t)) {
-            int &n_pv = t ? n_pv1 : n_pv0;
-            ok = mbar_wait(&bars->p_full[t], n_pv & 1, abort);
-            if (!ok) break;
-            ++n_pv;
-            tc_fence_after();
-            issue_pv(t, k);
-          }
-          if (more && active(k + 1, t)) issue_qk(t, k + 1);
+        issue_pv(k);
+        if (k + 2 < NT) {
+          ok = mbar_wait(&bars->k_full[t], ph ^ 1, abort);
+          if (!ok) break;
+          tc_fence_after();
+          issue_qk(k + 2);
         }
-        if (!ok) break;
-        tc_commit(&bars->v_empty[s]);
-        if (more) tc_commit(&bars->k_empty[(k + 1) & 1]);
       }
     }
   } else {
-    // ===== softmax / correction / epilogue: thread = (query row of either tile, half of the key columns)
-    // The tile index t is a run-time value on purpose: one compact copy of this code serves both
-    // tiles, which keeps the loop inside the instruction cache.
+    // ===== softmax / correction / epilogue: thread = (query row, half of the key columns), both streams
+    // The stream index t is a run-time value on purpose: one compact copy of this code serves both
+    // streams, which keeps the loop inside the instruction cache.
     const int a = (warp - 2) >> 2;  // column half: S columns [64a, 64a+64), O columns [64a, 64a+64)
     const int q = warp & 3;         // TMEM lane quarter this warp may touch
-    const int row = q * 32 + lane;  // row inside a 128-row query tile
+    const int row = q * 32 + lane;  // row inside the 128-row query tile
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
     const float c = p.scale_log2;
     float m_ref0 = -INFINITY, m_ref1 = -INFINITY, l_part0 = 0.f, l_part1 = 0.f;
-    int n_act0 = 0, n_act1 = 0;
     bool ok = true;
-    const int my_sub = (a * 64) / B;           // key sub-block this thread's columns belong to
+    const int my_sub = (a * 64) / B;             // key sub-block this thread's columns belong to
     const int col_in_sub = a * 64 - my_sub * B;  // first of its columns inside that sub-block
-    for (int kt = 0; kt < 2 * NT && ok; ++kt) {
-      const int k = kt >> 1, t = kt & 1;
+    const uint32_t my_bit = 1u << (row / B);     // query block of this row (uniform within a warp)
+    for (int k = 0; k < NT && ok; ++k) {
+      const int t = k & 1, n_act = k >> 1;
       const int nsub = min(SUBS, U - k * SUBS);
       // valid key columns, for this row, of the thread's two 32-column chunks
-      uint32_t tile_flags = 0;
       int lim0 = 0, lim1 = 0;
-      {
-        const uint32_t my_bit = 1u << (t * L::QBT + row / B);  // uniform within a warp
-#pragma unroll
-        for (int sub = 0; sub < SUBS; ++sub) {
-          if (sub < nsub) {
-            const uint32_t e = (uint32_t)uni[k * SUBS + sub];
-            tile_flags |= e >> 16;
-            if (sub == my_sub && ((e >> 16) & my_bit)) {
-              const int v = min(B, p.N - (int)(e & 0xffff) * B) - col_in_sub;
-              lim0 = max(0, min(32, v));
-              lim1 = max(0, min(32, v - 32));
-            }
-          }
+      if (my_sub < nsub) {
+        const uint32_t e = (uint32_t)uni[k * SUBS + my_sub];
+        if ((e >> 16) & my_bit) {
+          const int v = min(B, p.N - (int)(e & 0xffff) * B) - col_in_sub;
+          lim0 = max(0, min(32, v));
+          lim1 = max(0, min(32, v - 32));
         }
       }
-      if ((tile_flags & (tile_mask0 << (t * L::QBT))) == 0u) continue;
-      const int n_act = t ? n_act1 : n_act0;
       float m_ref = t ? m_ref1 : m_ref0;
       const uint32_t s_addr = lane_addr + t * 128 + a * 64;
       const uint32_t o_addr = lane_addr + 256 + t * 128 + a * 64;
@@ -386,7 +337,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         grow = true;
       }
       if (__any_sync(0xffffffffu, grow) && n_act > 0) {
-        // O_t must be quiescent: the latest PV of this tile has to be complete
+        // O_t must be quiescent: the latest PV of this stream has to be complete
         ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[t], (n_act - 1) & 1, abort));
         if (!ok) break;
         tc_fence_after();
@@ -434,59 +385,70 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       if (t) {
         m_ref1 = m_ref;
         l_part1 = l_new;
-        ++n_act1;
       } else {
         m_ref0 = m_ref;
         l_part0 = l_new;
-        ++n_act0;
       }
     }
-    // epilogue: each warpgroup writes its 64-dim half of both tiles' output rows
-#pragma unroll 1
-    for (int t = 0; t < 2; ++t) {
-      const int tok = row0 + t * 128 + row;
-      const bool valid_row = tok < p.N;
-      const int n_act = t ? n_act1 : n_act0;
-      const float m_ref = t ? m_ref1 : m_ref0;
-      const uint32_t o_addr = lane_addr + 256 + t * 128 + a * 64;
-      float *xrow = xch + (t * 2) * 128 + row;
-      float l = t ? l_part1 : l_part0;
-      if (ok && n_act > 0) {
-        xrow[a * 128] = l;  // the halves add their partial row sums
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->x_full[t][q]);
-        ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[t][q], n_act & 1, abort));
-        if (ok) l += xrow[(1 - a) * 128];
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[t], (n_act - 1) & 1, abort));
-      }
-      if (!ok) break;
+    // epilogue: merge the two streams; each warpgroup writes its 64-dim half of the output rows
+    const int n0 = (NT + 1) >> 1, n1 = NT >> 1;  // tiles per stream
+    const int tok = row0 + row;
+    const bool valid_row = tok < p.N;
+    float l0 = l_part0, l1 = l_part1;
+    if (ok && n0 > 0) {  // the column halves add their partial row sums (stream 0, then stream 1)
+      // (own slots, not the ones of the row maxima: a slow partner may still be reading those)
+      xch[512 + row + a * 128] = l_part0;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->x_full[0][q]);
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[0][q], n0 & 1, abort));
+      if (ok) l0 += xch[512 + row + (1 - a) * 128];
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[0], (n0 - 1) & 1, abort));
+    }
+    if (ok && n1 > 0) {
+      xch[768 + row + a * 128] = l_part1;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->x_full[1][q]);
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[1][q], n1 & 1, abort));
+      if (ok) l1 += xch[768 + row + (1 - a) * 128];
+      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[1], (n1 - 1) & 1, abort));
+    }
+    if (ok) {
       tc_fence_after();
+      const float m = fmaxf(m_ref0, m_ref1);
+      const float w0 = (n0 > 0 && m_ref0 > -INFINITY) ? ex2(m_ref0 - m) : 0.f;
+      const float w1 = (n1 > 0 && m_ref1 > -INFINITY) ? ex2(m_ref1 - m) : 0.f;
+      const float l = l0 * w0 + l1 * w1;
       const float inv = l > 0.f ? 1.f / l : 0.f;
+      const float f0 = w0 * inv, f1 = w1 * inv;
       uint16_t *orow = p.O + (long long)bidx * p.sb + (long long)hidx * p.sh + (long long)tok * p.sn + a * 64;
+      const uint32_t o_addr = lane_addr + 256 + a * 64;
 #pragma unroll 1
-      for (int ch = 0; ch < 2; ++ch) {
-        uint32_t v[32];
-        if (n_act > 0) {
-          tmem_ld32(o_addr + ch * 32, v);
-          tmem_wait_ld();
-        } else {
+      for (int ch = 0; ch < 4; ++ch) {  // 16 output dims at a time
+        uint32_t v0[16], v1[16];
+        if (n0 > 0) tmem_ld16(o_addr + ch * 16, v0);
+        if (n1 > 0) tmem_ld16(o_addr + 128 + ch * 16, v1);
+        tmem_wait_ld();
+        float o[16];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0u;
+        for (int i = 0; i < 16; ++i) {
+          o[i] = 0.f;
+          if (n0 > 0) o[i] = __uint_as_float(v0[i]) * f0;
+          if (n1 > 0) o[i] = fmaf(__uint_as_float(v1[i]), f1, o[i]);
         }
         if (valid_row) {
 #pragma unroll
-          for (int g4 = 0; g4 < 4; ++g4) {
-            uint4 o;
-            o.x = pack_bf16x2(__uint_as_float(v[g4 * 8 + 0]) * inv, __uint_as_float(v[g4 * 8 + 1]) * inv);
-            o.y = pack_bf16x2(__uint_as_float(v[g4 * 8 + 2]) * inv, __uint_as_float(v[g4 * 8 + 3]) * inv);
-            o.z = pack_bf16x2(__uint_as_float(v[g4 * 8 + 4]) * inv, __uint_as_float(v[g4 * 8 + 5]) * inv);
-            o.w = pack_bf16x2(__uint_as_float(v[g4 * 8 + 6]) * inv, __uint_as_float(v[g4 * 8 + 7]) * inv);
-            *reinterpret_cast<uint4 *>(orow + ch * 32 + g4 * 8) = o;
+          for (int g4 = 0; g4 < 2; ++g4) {
+            uint4 w;
+            w.x = pack_bf16x2(o[g4 * 8 + 0], o[g4 * 8 + 1]);
+            w.y = pack_bf16x2(o[g4 * 8 + 2], o[g4 * 8 + 3]);
+            w.z = pack_bf16x2(o[g4 * 8 + 4], o[g4 * 8 + 5]);
+            w.w = pack_bf16x2(o[g4 * 8 + 6], o[g4 * 8 + 7]);
+            *reinterpret_cast<uint4 *>(orow + ch * 16 + g4 * 8) = w;
           }
         }
       }
       if (a == 0 && valid_row && p.lse != nullptr)
-        p.lse[(size_t)r * p.N + tok] = l > 0.f ? (m_ref + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        p.lse[(size_t)r * p.N + tok] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
 
@@ -564,7 +526,7 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
   prm.N = g.N;
   prm.nb = g.nb;
   prm.idx_stride = g.idx_stride;
-  prm.n_ctas_per_head = (g.N + 255) / 256;
+  prm.n_ctas_per_head = (g.N + 127) / 128;
   prm.dense = dense ? 1 : 0;
   prm.scale_log2 = (float)(g.scale * 1.4426950408889634);
   ++*launches;
