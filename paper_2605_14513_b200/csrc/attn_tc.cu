@@ -218,27 +218,46 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       const uint64_t v_desc = smem_desc_sw128(smem_u32(Vs), 128 * 128, 1024);
       bool ok = true;
       auto keys_in = [&](int k) -> int { return min(SUBS, U - k * SUBS) * B; };
+      // every descriptor is formed once, outside the loop: issuing a tile is 8 back-to-back MMAs
+      uint64_t qd[8], kd[2][8], vd[2][8];
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        qd[ks] = q_desc + ((ks >> 2) * 1024 + (ks & 3) * 2);
+        kd[0][ks] = k_desc + ((ks >> 2) * 1024 + (ks & 3) * 2);
+        kd[1][ks] = kd[0][ks] + (L::TILE_BYTES >> 4);
+        vd[0][ks] = v_desc + ks * 128;
+        vd[1][ks] = vd[0][ks] + (L::TILE_BYTES >> 4);
+      }
       auto issue_qk = [&](int k) {  // S_t = Q K_k^T, t = k & 1; K_k sits in stage t
         const int t = k & 1;
-        const uint64_t b0 = k_desc + (uint64_t)(t * (L::TILE_BYTES >> 4));
         const uint32_t d = tmem + t * 128;
         const uint32_t idesc = keys_in(k) == 128 ? idesc_qk_full : idesc_qk_half;
+        if (t == 0) {
+          mma_ss(d, qd[0], kd[0][0], idesc, 0u);
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          mma_ss(d, q_desc + ((ks >> 2) * 1024 + (ks & 3) * 2), b0 + ((ks >> 2) * 1024 + (ks & 3) * 2), idesc, ks > 0 ? 1u : 0u);
+          for (int ks = 1; ks < 8; ++ks) mma_ss(d, qd[ks], kd[0][ks], idesc, 1u);
+        } else {
+          mma_ss(d, qd[0], kd[1][0], idesc, 0u);
+#pragma unroll
+          for (int ks = 1; ks < 8; ++ks) mma_ss(d, qd[ks], kd[1][ks], idesc, 1u);
+        }
         tc_commit(&bars->s_full[t]);
         tc_commit(&bars->k_empty[t]);
       };
       auto issue_pv = [&](int k) {  // O_t (+)= P_t V_k
         const int t = k & 1;
-        const uint64_t b0 = v_desc + (uint64_t)(t * (L::TILE_BYTES >> 4));
         const uint32_t d = tmem + 256 + t * 128, pa = tmem + t * 128;
-        mma_ts(d, pa, b0, idesc_pv, k >= 2 ? 1u : 0u);
+        const int ksteps = keys_in(k) / 16;
+        if (t == 0) {
+          mma_ts(d, pa, vd[0][0], idesc_pv, k >= 2 ? 1u : 0u);
 #pragma unroll
-        for (int ks = 1; ks < 4; ++ks) mma_ts(d, pa + ks * 8, b0 + ks * 128, idesc_pv, 1u);
-        if (keys_in(k) == 128) {
+          for (int ks = 1; ks < 8; ++ks)
+            if (ks < ksteps) mma_ts(d, pa + ks * 8, vd[0][ks], idesc_pv, 1u);
+        } else {
+          mma_ts(d, pa, vd[1][0], idesc_pv, k >= 2 ? 1u : 0u);
 #pragma unroll
-          for (int ks = 4; ks < 8; ++ks) mma_ts(d, pa + ks * 8, b0 + ks * 128, idesc_pv, 1u);
+          for (int ks = 1; ks < 8; ++ks)
+            if (ks < ksteps) mma_ts(d, pa + ks * 8, vd[1][ks], idesc_pv, 1u);
         }
         tc_commit(&bars->pv_done[t]);
         tc_commit(&bars->v_empty[t]);
