@@ -3,21 +3,24 @@
 // cumulative-mass set of Observation I).  Importance = row softmax of the block-pooled Q.K^T scores.
 //
 // One CTA owns TI = 16 query blocks of one head.  Phase 1 is a register-tiled fp64 contraction of
-// the pooled means (each thread 4 query blocks x 4 key blocks, key means staged through shared
-// memory 256 blocks x 32 dims at a time) into a shared-memory tile of scores.  Phase 2 gives each
+// the pooled means (each thread 8 query blocks x 4 key blocks, key means staged through shared
+// memory 512 blocks x 16 dims at a time with the next stage's loads in flight) into a shared-memory
+// tile of scores.  Phase 2 gives each
 // warp two rows: two-pass softmax, then top-p WITHOUT a sort: the kept set is {p > theta} plus the
 // lowest-index ties at theta, where theta is the largest element value whose ">= theta" mass still
 // reaches tau -- found by a 62-step bit-wise search over the IEEE-754 pattern of p (positive
 // doubles order like their bit patterns).  Everything is fp64 so the integer outputs (bit mask,
 // ascending index list, count) agree with a plain fp64 sort-and-accumulate reference except when
 // the cumulative mass is within rounding (1e-15) of tau.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace heart {
 
 constexpr int TI = 16;    // query blocks per CTA
-constexpr int TJ = 256;   // key blocks per staged pass
-constexpr int TD = 32;    // dims per staged chunk
+constexpr int TJ = 512;   // key blocks per staged pass
+constexpr int TD = 16;    // dims per staged chunk
 constexpr int KLD = TD + 1;
 
 __device__ __forceinline__ double warp_sum(double v) {
@@ -61,51 +64,74 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
     Qs[e] = v;
   }
 
-  // ---- phase 1: S[i][J] = scale * <Qp[I0+i], Kp[J]>
-  const int ig = warp & 3, jh = warp >> 2;
-  for (int jc = 0; jc < nb; jc += TJ) {
-    double acc[4][4];
+  // ---- phase 1: S[i][J] = scale * <Qp[I0+i], Kp[J]>.  Each thread owns 8 query blocks x 4 key blocks;
+  // the key means are staged 512 blocks x 16 dims at a time, and the loads of the next stage are in
+  // flight (in registers) while the current one is multiplied.
+  const int rg = tid >> 7, cl = tid & 127;
+  constexpr int PER = (TJ * TD) / 256;  // staged values per thread = 32
+  const int n_jc = (nb + TJ - 1) / TJ, n_stage = n_jc * (kD / TD);
+  double pre[PER];
+  auto fetch = [&](int stage) {
+    const int jc = (stage / (kD / TD)) * TJ, dc = (stage % (kD / TD)) * TD;
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int m = 0; m < 4; ++m) acc[a][m] = 0.0;
-    for (int dc = 0; dc < kD; dc += TD) {
-      __syncthreads();
-      {  // all 32 loads of this thread in flight before the first use
-        double v[(TJ * TD) / 256];
-#pragma unroll
-        for (int k = 0; k < (TJ * TD) / 256; ++k) {
-          const int e = tid + 256 * k, J = jc + e / TD;
-          v[k] = (J < nb) ? bk[(size_t)J * kD + dc + (e % TD)] : 0.0;
-        }
-#pragma unroll
-        for (int k = 0; k < (TJ * TD) / 256; ++k) {
-          const int e = tid + 256 * k, row = e / TD, J = jc + row;
-          // full blocks: 1/block is a power of two, so the product equals the division exactly
-          Ks[row * KLD + (e % TD)] = (J == nb - 1) ? v[k] / (double)last_cnt : v[k] * inv_block;
-        }
-      }
-      __syncthreads();
-#pragma unroll 8
-      for (int dd = 0; dd < TD; ++dd) {
-        double q[4], k[4];
-#pragma unroll
-        for (int a = 0; a < 4; ++a) q[a] = Qs[(ig * 4 + a) * kD + dc + dd];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) k[m] = Ks[(jh * 128 + lane + 32 * m) * KLD + dd];
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-          for (int m = 0; m < 4; ++m) acc[a][m] = fma(q[a], k[m], acc[a][m]);
-      }
+    for (int k = 0; k < PER; ++k) {
+      const int e = tid + 256 * k, J = jc + e / TD;
+      pre[k] = (J < nb) ? bk[(size_t)J * kD + dc + (e % TD)] : 0.0;
     }
+  };
+  fetch(0);
+  double acc[8][4];
+  for (int stage = 0; stage < n_stage; ++stage) {
+    const int jc = (stage / (kD / TD)) * TJ, dc = (stage % (kD / TD)) * TD;
+    if (dc == 0) {
 #pragma unroll
-    for (int a = 0; a < 4; ++a)
+      for (int a = 0; a < 8; ++a)
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        const int J = jc + jh * 128 + lane + 32 * m;
-        if (J < NBP) S[(ig * 4 + a) * NBP + J] = acc[a][m] * scale;
+        for (int m = 0; m < 4; ++m) acc[a][m] = 0.0;
+    }
+    __syncthreads();  // the previous stage has been consumed
+#pragma unroll
+    for (int k = 0; k < PER; ++k) {
+      const int e = tid + 256 * k, row = e / TD, J = jc + row;
+      // full blocks: 1/block is a power of two, so the product equals the division exactly
+      Ks[row * KLD + (e % TD)] = (J == nb - 1) ? pre[k] / (double)last_cnt : pre[k] * inv_block;
+    }
+    __syncthreads();
+    if (stage + 1 < n_stage) fetch(stage + 1);
+    // column groups of 128 key blocks that exist in this pass (the last pass is usually short)
+    const int nm = min(4, (nb - jc + 127) >> 7);
+    auto multiply = [&](auto NM) {
+      constexpr int kNm = decltype(NM)::value;
+#pragma unroll 4
+      for (int dd = 0; dd < TD; ++dd) {
+        double q[8], k4[kNm];
+#pragma unroll
+        for (int a = 0; a < 8; ++a) q[a] = Qs[(rg * 8 + a) * kD + dc + dd];
+#pragma unroll
+        for (int m = 0; m < kNm; ++m) k4[m] = Ks[(cl + 128 * m) * KLD + dd];
+#pragma unroll
+        for (int a = 0; a < 8; ++a)
+#pragma unroll
+          for (int m = 0; m < kNm; ++m) acc[a][m] = fma(q[a], k4[m], acc[a][m]);
       }
+    };
+    if (nm == 4)
+      multiply(std::integral_constant<int, 4>{});
+    else if (nm == 3)
+      multiply(std::integral_constant<int, 3>{});
+    else if (nm == 2)
+      multiply(std::integral_constant<int, 2>{});
+    else
+      multiply(std::integral_constant<int, 1>{});
+    if (dc == kD - TD) {
+#pragma unroll
+      for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          const int J = jc + cl + 128 * m;
+          if (J < NBP) S[(rg * 8 + a) * NBP + J] = acc[a][m] * scale;
+        }
+    }
   }
   __syncthreads();
 
@@ -146,14 +172,57 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
     long long theta = 0;
     int m_ties = 0;
     if (!keep_all) {
-      for (int bit = 61; bit >= 0; --bit) {
-        const long long cand = theta | (1LL << bit);
-        double g = 0.0;
+      // Full-width rounds for the exponent and the top mantissa bits ...
+      auto mass_at_least = [&](long long cand) -> double {
+        double g0 = 0.0, g1 = 0.0, g2 = 0.0, g3 = 0.0;  // fixed 4-way split: same order on every run
 #pragma unroll
-        for (int j = 0; j < NJ; ++j)
-          if (__double_as_longlong(p[j]) >= cand) g += p[j];
-        g = warp_sum(g);
-        if (g >= t) theta = cand;
+        for (int j = 0; j < NJ; j += 4) {
+          if (__double_as_longlong(p[j]) >= cand) g0 += p[j];
+          if (j + 1 < NJ && __double_as_longlong(p[j + 1]) >= cand) g1 += p[j + 1];
+          if (j + 2 < NJ && __double_as_longlong(p[j + 2]) >= cand) g2 += p[j + 2];
+          if (j + 3 < NJ && __double_as_longlong(p[j + 3]) >= cand) g3 += p[j + 3];
+        }
+        return warp_sum((g0 + g1) + (g2 + g3));
+      };
+      constexpr int kSplit = 48;  // bits [kSplit, 62) are searched over all blocks
+      for (int bit = 61; bit >= kSplit; --bit) {
+        const long long cand = theta | (1LL << bit);
+        if (mass_at_least(cand) >= t) theta = cand;
+      }
+      // ... then only the blocks whose pattern shares that prefix can still decide the remaining bits:
+      // they are compacted (through this row's no longer needed score slots) and the other 48 rounds
+      // run on at most two candidates per lane.  Blocks above the prefix enter as one constant.
+      const long long hi = theta >> kSplit;
+      double *scr = S + i * NBP;
+      double ab0 = 0.0, ab1 = 0.0;
+      int n_cand = 0;
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < NJ; ++j) {
+        const long long kh = __double_as_longlong(p[j]) >> kSplit;
+        if (kh > hi) {
+          if (j & 1) ab1 += p[j]; else ab0 += p[j];
+        }
+        const bool is_c = (kh == hi) && (j * 32 + lane < nb);
+        const unsigned bal = __ballot_sync(0xffffffffu, is_c);
+        if (is_c) scr[n_cand + __popc(bal & lt_mask)] = p[j];
+        n_cand += __popc(bal);
+      }
+      const double mass_above = warp_sum(ab0 + ab1);
+      __syncwarp();
+      if (n_cand <= 64) {
+        const double c0 = (lane < n_cand) ? scr[lane] : 0.0, c1 = (lane + 32 < n_cand) ? scr[lane + 32] : 0.0;
+        const long long k0 = __double_as_longlong(c0), k1 = __double_as_longlong(c1);
+        for (int bit = kSplit - 1; bit >= 0; --bit) {
+          const long long cand = theta | (1LL << bit);
+          const double g = mass_above + warp_sum((k0 >= cand ? c0 : 0.0) + (k1 >= cand ? c1 : 0.0));
+          if (g >= t) theta = cand;
+        }
+      } else {  // many near-equal blocks: keep searching over all of them
+        for (int bit = kSplit - 1; bit >= 0; --bit) {
+          const long long cand = theta | (1LL << bit);
+          if (mass_at_least(cand) >= t) theta = cand;
+        }
       }
       double above = 0.0;
       int nties = 0;
