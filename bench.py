@@ -111,7 +111,7 @@ def run_ours(args, rank, world):
     import torch
     import torch.distributed as dist
 
-    from paper_2605_14513_b200 import heart, inputs
+    from paper_2605_14513_b200 import heart, inputs, replicas
 
     heart.lib()  # fails loudly if the CUDA library is missing
     local = int(os.environ.get("LOCAL_RANK", 0))
@@ -145,8 +145,7 @@ def run_ours(args, rank, world):
         heart.heart_step(cfg, Q, Kt, V, delta, tau, st, O, ws, drift_out=drift, refresh_out=refresh)
 
     def barrier():
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     for t in range(W):
@@ -171,10 +170,7 @@ def run_ours(args, rank, world):
     clocks = sampler.stop() if sampler else None
     total_ms = ev[0][0].elapsed_time(ev[-1][1])
     assert heart.heart_get_status(ws) == 0
-    if world > 1:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = replicas.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / K
 
     # ---- per-stage pass: the same K steps as three C-ABI calls, one event pair per call.  Nothing here
@@ -227,12 +223,9 @@ def run_ours(args, rank, world):
         b_.record()
         barrier()
         e2e_ms = a.elapsed_time(b_) / Ke
-        if world > 1:
-            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt.item())
+        e2e_ms = replicas.max_over_ranks(e2e_ms, dev)
         tensor_bytes = 2 * wl.R * wl.N * wl.D
-        e2e = {"value": e2e_ms / world, "unit": "ms", "steps": Ke, "h2d_bytes_per_step": 3 * tensor_bytes,
+        e2e = {"value": replicas.job_ms_per_layer_step(e2e_ms, world), "unit": "ms", "steps": Ke, "h2d_bytes_per_step": 3 * tensor_bytes,
                "d2h_bytes_per_step": tensor_bytes + 9 * wl.R,
                "api": "heart_step_host (pinned host Q/K/V in, O + drift + refresh out)"}
         del host_in, staging
@@ -248,7 +241,7 @@ def run_ours(args, rank, world):
                     "flops_per_launch": flops_step, "ms_per_launch": ms_attn}
         hbm = stats_bytes / (ms_drift * 1e-3) / 1e9
         out = {
-            "metric": METRIC, "value": ms_per_step / world, "unit": "ms", "n_gpus": world, "steps": K, "warmup": W,
+            "metric": METRIC, "value": replicas.job_ms_per_layer_step(ms_per_step, world), "unit": "ms", "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "grid": list(wl.grid), "D": wl.D,
