@@ -266,3 +266,28 @@ def test_full_size_configs(heart, oracle, name, steps, n_sample):
     assert ex_rows <= max(1, int(1e-3 * total_rows)) and ex_flags == 0
     dens = pair.ost.kv_cnt.mean() / wl.n_blocks
     assert 0.03 < dens < 0.5
+
+
+# ------------------------------------------------------------------ size limits
+def test_maximum_block_count(heart, oracle):
+    """n_b = 1024 (the largest supported): N = 64 * 1024 - 9 tokens at block 64, one head.  Masks and
+    decisions in full, attention on sampled query blocks."""
+    wl = inputs.small_workload(H=1, grid=(1, 1, 64 * 1024 - 9), block=64, seed=13, tau=[0.9], eps=[0.05],
+                               delta=[0.01])
+    assert wl.n_blocks == heart.MAX_BLOCKS
+    pair = Pair(wl, heart, oracle)
+    seen, ex_rows, ex_flags = run_sweep(pair, 2, full_attention=False, n_sample=6, seed=2)
+    assert ex_rows == 0 and ex_flags == 0
+    cfg = heart.make_config(1, 1, 64 * 1024 + 1, 64)  # one block too many
+    assert heart.workspace_bytes(cfg) == 0
+
+
+@pytest.mark.parametrize("N,block", [(1, 64), (63, 64), (65, 128), (129, 128)])
+def test_tiny_token_counts(heart, oracle, N, block):
+    """Fewer tokens than a block, one token more than a block: ragged tiles everywhere."""
+    wl = inputs.small_workload(H=2, grid=(1, 1, N), block=block, seed=N, tau=[0.7, 1.0], eps=[0.3, 0.3],
+                               delta=[0.0, 0.0])
+    pair = Pair(wl, heart, oracle)
+    seen, ex_rows, ex_flags = run_sweep(pair, 2)
+    assert np.all(seen[0] == 1) and np.all(seen[1] == 1)  # delta = 0 and moving inputs: always refresh
+    assert ex_rows == 0 and ex_flags == 0
