@@ -38,7 +38,7 @@ def parse():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="wan1.3b-480p")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cpu-sample-rows", type=int, default=64, help="query blocks the CPU oracle attends per step")
+    ap.add_argument("--cpu-sample-rows", type=int, default=384, help="query blocks the CPU oracle attends per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
