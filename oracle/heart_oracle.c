@@ -463,3 +463,30 @@ void oracle_step(const uint16_t *Q, const uint16_t *K, const uint16_t *V, int B,
   free(mq);
   free(mk);
 }
+
+/* ---------------------------------------------------------------------------
+ * Block-mask IoU between two steps (Observation I, adjacent-step mask
+ * similarity: |M_a AND M_b| / |M_a OR M_b|), taken over the retained
+ * (query block, key block) pairs of each head.  mask_* are [R][nb][W] bit
+ * masks as written by oracle_predict_mask.  Two empty masks give IoU = 1.
+ * counts (optional) receives [R][2] = (intersection, union).
+ * ------------------------------------------------------------------------ */
+void oracle_mask_iou(const uint32_t *mask_a, const uint32_t *mask_b, int R, int nb, double *iou,
+                     int64_t *counts) {
+  int W = (nb + 31) / 32;
+  for (int r = 0; r < R; ++r) {
+    int64_t inter = 0, uni = 0;
+    for (int I = 0; I < nb; ++I)
+      for (int J = 0; J < nb; ++J) {
+        size_t w = ((size_t)r * nb + I) * W + (J >> 5);
+        int a = (mask_a[w] >> (J & 31)) & 1, b = (mask_b[w] >> (J & 31)) & 1;
+        inter += a & b;
+        uni += a | b;
+      }
+    iou[r] = uni ? (double)inter / (double)uni : 1.0;
+    if (counts) {
+      counts[2 * r] = inter;
+      counts[2 * r + 1] = uni;
+    }
+  }
+}

@@ -217,3 +217,14 @@ def step(Q, K, V, delta, tau, st: State, scale=0.0, gate_lo=0.0, gate_hi=1.0, fl
                       _p(st.kv_idx), _p(st.kv_cnt), st.idx_stride, _p(O), _p(lse), _p(drift),
                       _p(refresh))
     return O, lse, drift, refresh
+
+
+def mask_iou(mask_a, mask_b, nb):
+    """Block-mask IoU per head between two [R, nb, W] bit masks -> (iou[R], counts[R, 2])."""
+    mask_a = np.ascontiguousarray(mask_a, np.uint32)
+    mask_b = np.ascontiguousarray(mask_b, np.uint32)
+    R = mask_a.shape[0]
+    iou = np.empty(R, np.float64)
+    counts = np.empty((R, 2), np.int64)
+    lib().oracle_mask_iou(_p(mask_a), _p(mask_b), R, int(nb), _p(iou), _p(counts))
+    return iou, counts

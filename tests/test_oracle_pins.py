@@ -537,3 +537,42 @@ def test_tiny_config_refresh_pattern(oracle):
     assert np.array_equal(st.kv_cnt[0], cnt0[0])  # reused head keeps its mask
     dens = st.kv_cnt.mean(axis=1) / wl.n_blocks
     assert np.all(dens > 0.1) and np.all(dens < 0.8)
+
+
+# ----------------------------------------------------------------------------- diagnostics
+def test_mask_iou_closed_forms(oracle):
+    nb, W = 40, 2
+    a = np.zeros((3, nb, W), np.uint32)
+    b = np.zeros((3, nb, W), np.uint32)
+    # head 0: identical masks (every row keeps blocks 0..9) -> IoU 1
+    a[0, :, 0] = b[0, :, 0] = (1 << 10) - 1
+    # head 1: A keeps blocks 0..9, B keeps 5..14 -> |A&B| = 5, |A|B| = 15 per row -> 1/3
+    a[1, :, 0] = (1 << 10) - 1
+    b[1, :, 0] = ((1 << 15) - 1) ^ ((1 << 5) - 1)
+    # head 2: disjoint, B in the second word (blocks 32..39) -> 0
+    a[2, :, 0] = 0xff
+    b[2, :, 1] = 0xff
+    iou, counts = oracle.mask_iou(a, b, nb)
+    assert np.array_equal(iou, [1.0, 5.0 / 15.0, 0.0])
+    assert np.array_equal(counts, [[10 * nb, 10 * nb], [5 * nb, 15 * nb], [0, 16 * nb]])
+    # both empty -> 1 by convention; symmetric
+    z = np.zeros_like(a)
+    assert np.array_equal(oracle.mask_iou(z, z, nb)[0], [1.0, 1.0, 1.0])
+    assert np.array_equal(oracle.mask_iou(b, a, nb)[0], iou)
+
+
+def test_mask_iou_of_predicted_masks_drops_with_drift(oracle):
+    """Small drift keeps the predicted mask (IoU near 1), large drift changes it: the relation the
+    paper's reuse rule relies on, on the synthetic tensors."""
+    wl = inputs.small_workload(H=2, grid=(3, 10, 14), block=64, seed=17, eps=[0.002, 0.6], tau=[0.9, 0.9])
+    seq = inputs.Sequence(wl)
+    Q, K, _ = (inputs.bits(x) for x in seq.bf16())
+    s0 = oracle.State(1, 2, wl.N, 128, 64)
+    oracle.predict_mask(Q, K, 64, wl.tau, s0)
+    seq.advance()
+    Q1, K1, _ = (inputs.bits(x) for x in seq.bf16())
+    s1 = oracle.State(1, 2, wl.N, 128, 64)
+    oracle.predict_mask(Q1, K1, 64, wl.tau, s1)
+    iou, _ = oracle.mask_iou(s0.mask_bits, s1.mask_bits, wl.n_blocks)
+    full = oracle.full_token_drift(Q, K, Q1, K1)
+    assert iou[0] > 0.9 and iou[1] < iou[0] and full[1] > 50 * full[0]
