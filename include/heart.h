@@ -174,6 +174,26 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
 int heart_drift_static(const heart_config *cfg, const void *Q, const void *K, const double *delta,
                        heart_state *st, double *drift_out, uint8_t *refresh_out, heart_stream_t stream);
 
+/* ---- Analysis quantities (not on the layer-step path; nothing else reads their results) ---- */
+
+/* Full-token drift between two steps of the same layer -- Eq. full-token drift, the costly
+ * reference that the mean-pooled drift of heart_drift approximates (TMR section):
+ *   drift_out[r] = (1/N) sum_i ( ||Qa[r,i]-Qb[r,i]||_1 + ||Ka[r,i]-Kb[r,i]||_1 ),  fp64 [R].
+ * Qa, Ka (the cached step) and Qb, Kb (the current step) are bf16 with the layout cfg gives.
+ * One streaming pass over the four tensors; uses the workspace as scratch (a later heart_drift or
+ * heart_predict_mask rewrites what it needs); reads and writes no TMR state. */
+int heart_full_token_drift(const heart_config *cfg, const void *Qa, const void *Ka, const void *Qb,
+                           const void *Kb, double *drift_out, void *workspace, heart_stream_t stream);
+
+/* Block-mask IoU between two steps -- Observation I (adjacent-step mask similarity), taken over the
+ * retained (query block, key block) pairs of each head:
+ *   iou_out[r] = |A_r AND B_r| / |A_r OR B_r|   (1 when both masks are empty), fp64 [R].
+ * mask_a, mask_b: [R, n_b, W] bit masks in the mask_bits layout of heart_state (bits at J >= n_b
+ * must be zero, as heart_predict_mask leaves them).  counts_out: optional int64 [R, 2] =
+ * (intersection, union) pair counts, or NULL. */
+int heart_mask_iou(const heart_config *cfg, const uint32_t *mask_a, const uint32_t *mask_b,
+                   double *iou_out, int64_t *counts_out, heart_stream_t stream);
+
 /* Synchronises `stream`, reads the workspace status word into *code_out (host) and clears it.
  * The only call that blocks. */
 int heart_get_status(void *workspace, heart_stream_t stream, int32_t *code_out /* host */);

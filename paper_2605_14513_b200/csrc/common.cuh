@@ -83,4 +83,11 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,
                              float *lse, int32_t *status, cudaStream_t s, int *launches);
 
+cudaError_t launch_token_drift(const Geom &g, const void *Qa, const void *Ka, const void *Qb,
+                               const void *Kb, double *partial, double *drift_out, cudaStream_t s,
+                               int *launches);
+int token_drift_chunks(const Geom &g, int *rows_per_cta);
+cudaError_t launch_mask_iou(const Geom &g, const uint32_t *A, const uint32_t *B, double *iou,
+                            long long *counts, cudaStream_t s, int *launches);
+
 }  // namespace heart

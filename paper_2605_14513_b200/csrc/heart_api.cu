@@ -212,6 +212,39 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
   return HEART_OK;
 }
 
+int heart_full_token_drift(const heart_config *cfg, const void *Qa, const void *Ka, const void *Qb,
+                           const void *Kb, double *drift_out, void *workspace, heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  if (!Qa || !Ka || !Qb || !Kb || !drift_out || !workspace) return HEART_ERR_INVALID;
+  if (!aligned16(Qa) || !aligned16(Ka) || !aligned16(Qb) || !aligned16(Kb) ||
+      (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return HEART_ERR_INVALID;
+  Workspace w = carve(g, workspace);
+  int rows = 0;
+  const size_t need = (size_t)g.R * token_drift_chunks(g, &rows);  // partials live in the block-sum area
+  if (need > 2 * (size_t)g.R * g.nb * kD) return HEART_ERR_INVALID;
+  g_launches = 0;
+  cudaError_t e = launch_token_drift(g, Qa, Ka, Qb, Kb, w.bsum, drift_out,
+                                     static_cast<cudaStream_t>(stream), &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "token_drift");
+  return HEART_OK;
+}
+
+int heart_mask_iou(const heart_config *cfg, const uint32_t *mask_a, const uint32_t *mask_b,
+                   double *iou_out, int64_t *counts_out, heart_stream_t stream) {
+  Geom g;
+  int rc = make_geom(cfg, &g);
+  if (rc != HEART_OK) return rc;
+  if (!mask_a || !mask_b || !iou_out) return HEART_ERR_INVALID;
+  g_launches = 0;
+  cudaError_t e = launch_mask_iou(g, mask_a, mask_b, iou_out, reinterpret_cast<long long *>(counts_out),
+                                  static_cast<cudaStream_t>(stream), &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "mask_iou");
+  return HEART_OK;
+}
+
 int heart_get_status(void *workspace, heart_stream_t stream, int32_t *code_out) {
   if (!workspace || !code_out) return HEART_ERR_INVALID;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

@@ -23,7 +23,7 @@ MAX_BLOCKS = 1024
 SYMBOLS = (
     "heart_workspace_bytes", "heart_state_reset", "heart_drift", "heart_predict_mask",
     "heart_block_sparse_attn", "heart_step", "heart_step_host", "heart_get_status", "heart_strerror",
-    "heart_last_launch_count", "heart_drift_static",
+    "heart_last_launch_count", "heart_drift_static", "heart_full_token_drift", "heart_mask_iou",
 )
 
 
@@ -72,6 +72,10 @@ def lib():
         l.heart_get_status.argtypes = [vp, vp, C.POINTER(C.c_int32)]
         l.heart_drift_static.argtypes = [C.POINTER(Config), vp, vp, vp, C.POINTER(StateStruct), vp, vp, vp]
         l.heart_drift_static.restype = C.c_int
+        l.heart_full_token_drift.argtypes = [C.POINTER(Config)] + [vp] * 7
+        l.heart_full_token_drift.restype = C.c_int
+        l.heart_mask_iou.argtypes = [C.POINTER(Config)] + [vp] * 5
+        l.heart_mask_iou.restype = C.c_int
         for fn in ("heart_state_reset", "heart_drift", "heart_predict_mask", "heart_block_sparse_attn",
                    "heart_step", "heart_step_host", "heart_get_status"):
             getattr(l, fn).restype = C.c_int
@@ -186,6 +190,20 @@ def heart_drift_static(cfg, Q, K, delta, st: State, drift_out=None, refresh_out=
     16 MiB array (shapes that need more raise ERR_TOO_LARGE).  Calls on one device must not overlap."""
     _check(lib().heart_drift_static(C.byref(cfg), _ptr(Q), _ptr(K), _ptr(delta), C.byref(st.struct),
                                     _ptr(drift_out), _ptr(refresh_out), _stream()))
+
+
+def heart_full_token_drift(cfg, Qa, Ka, Qb, Kb, drift_out, ws):
+    """Full-token drift (Eq. full-token drift) between a cached step (Qa, Ka) and the current one
+    (Qb, Kb) into drift_out [R] fp64."""
+    _check(lib().heart_full_token_drift(C.byref(cfg), _ptr(Qa), _ptr(Ka), _ptr(Qb), _ptr(Kb), _ptr(drift_out),
+                                        _ptr(ws), _stream()))
+
+
+def heart_mask_iou(cfg, mask_a, mask_b, iou_out, counts_out=None):
+    """Block-mask IoU per head between two [R, n_b, W] bit masks (Observation I) into iou_out [R] fp64;
+    counts_out: optional int64 [R, 2] = (intersection, union)."""
+    _check(lib().heart_mask_iou(C.byref(cfg), _ptr(mask_a), _ptr(mask_b), _ptr(iou_out), _ptr(counts_out),
+                                _stream()))
 
 
 def heart_get_status(ws) -> int:
