@@ -576,3 +576,34 @@ def test_mask_iou_of_predicted_masks_drops_with_drift(oracle):
     iou, _ = oracle.mask_iou(s0.mask_bits, s1.mask_bits, wl.n_blocks)
     full = oracle.full_token_drift(Q, K, Q1, K1)
     assert iou[0] > 0.9 and iou[1] < iou[0] and full[1] > 50 * full[0]
+
+
+def test_full_token_drift_bounds_the_interaction_change(oracle):
+    """Stability bound of the appendix: the mean absolute change of the scaled query-key logits is
+    at most max(B_q, B_k)/sqrt(D) times the full-token drift -- with equality when the keys are a
+    constant vector of magnitude B_k >= B_q that does not move and every query coordinate grows."""
+    rs = np.random.RandomState(21)
+    R, N, D = 2, 24, 16
+    # general case: inequality
+    Qa, fa = rand_bf16(rs, (R, N, D))
+    Ka, ka = rand_bf16(rs, (R, N, D))
+    Qb, fb = rand_bf16(rs, (R, N, D))
+    Kb, kb = rand_bf16(rs, (R, N, D))
+    d = oracle.full_token_drift(Qa, Ka, Qb, Kb)
+    for r in range(R):
+        ga = fa[r] @ ka[r].T / math.sqrt(D)
+        gb = fb[r] @ kb[r].T / math.sqrt(D)
+        Bq = max(np.abs(fa[r]).max(), np.abs(fb[r]).max())
+        Bk = max(np.abs(ka[r]).max(), np.abs(kb[r]).max())
+        assert np.abs(gb - ga).mean() <= max(Bq, Bk) / math.sqrt(D) * d[r] + 1e-12
+    # equality case (all values exactly representable in bf16)
+    qa = np.round(rs.uniform(-1, 1, (R, N, D)) * 8) / 8.0
+    inc = np.round(rs.uniform(0, 1, (R, N, D)) * 8) / 8.0
+    k = np.full((R, N, D), 2.0)
+    A, _ = bf16_bits(qa)
+    Bm, _ = bf16_bits(qa + inc)
+    Kc, _ = bf16_bits(k)
+    d = oracle.full_token_drift(A, Kc, Bm, Kc)
+    for r in range(R):
+        delta_qk = np.abs((qa[r] + inc[r]) @ k[r].T - qa[r] @ k[r].T).mean() / math.sqrt(D)
+        assert np.isclose(delta_qk, 2.0 / math.sqrt(D) * d[r], rtol=1e-13)
