@@ -2,25 +2,30 @@
 //
 // One CTA owns one 128-row query tile of one head: one query block of 128 tokens, or two query
 // blocks of 64 whose lists are merged into an ascending union (one flag bit per query block; rows of
-// the half that does not list a key block see -inf there).  Keys are processed 128 at a time: a key
-// tile is one 128-token block or two 64-token blocks of the union.
+// the half that does not list a key block see -inf there).  Keys are processed 64 at a time: a "key
+// step" is one 64-token block, or one half of a 128-token block.
 //
-// The key tiles are dealt to two independent streams (even / odd tile index).  Each stream keeps its
-// own running max, row sum and output accumulator and the two are merged at the end, so the softmax of
-// one stream overlaps the MMAs of the other (ping-pong) although both work for the same query rows.
+// The key steps are dealt to two independent streams (even / odd step index).  Each stream keeps
+// its own running max, row sum and output accumulator (merged at the end) and is served by its own
+// softmax warpgroup, one thread per query row, so the two warpgroups run out of phase: while one
+// computes exponentials the other waits, loads scores or takes maxima, and the special-function
+// unit -- the scarcest resource of this kernel -- stays busy.  Each stream double-buffers its scores
+// in tensor memory: S of the stream's next step is computed while the softmax works on the current
+// one, so the serial chain softmax -> P V -> Q K^T -> softmax is off the critical path.
 //
-// Warp roles (320 threads):
-//   warp 0      TMA producer: the Q tile once, then the listed K and V blocks through shared-memory
-//               rings (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers).
-//   warp 1      MMA issuer (one lane): S_t = Q K^T into tensor memory (tcgen05.mma, operands in shared
-//               memory), O_t += P_t V with P_t read from tensor memory.
-//   warps 2-9   softmax: both warpgroups work on the stream whose scores are ready, warpgroup a on key
-//               columns [64a, 64a+64); thread = (query row, column half).  It reads its half of the S
-//               row from tensor memory, the two halves exchange their row maxima through shared
-//               memory, it keeps the running max / partial sum, writes P (bf16) back over S,
-//               rescales its half of O only when the max grew by more than 2^8, and at the end merges
-//               the two streams and writes its half of O (and lse).
-// Tensor memory (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P_t aliases S_t.
+// Warp roles (352 threads):
+//   warp 0      TMA producer for Q (once) and K, through a four-stage shared-memory ring
+//               (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers).
+//   warp 1      MMA issuer (one lane): S_h = Q K_h^T into tensor memory (tcgen05.mma, operands in
+//               shared memory) and O_t += P_h V_h with P_h read from tensor memory.
+//   warps 2-5   softmax warpgroup of stream 0; warps 6-9 of stream 1.  Per key step a thread reads
+//               its row of S (64 columns), takes the max, rescales its row of O only when the max
+//               grew by more than 2^8, writes P = 2^(s*scale*log2e - m) as bf16 over the first half
+//               of the S buffer and adds the row sum.  At the end the two warpgroups exchange
+//               (max, sum), and warpgroup t writes output dims [64t, 64t+64) of every row (and lse).
+//   warp 10     TMA producer for V (its own ring: V_h is needed four key steps later than K_h).
+// Tensor memory (512 columns): O_0 | O_1 | S[4]  =  128 + 128 + 4 x 64; key step h uses S[h & 3]
+// (stream h & 1, buffer (h >> 1) & 1) and shared-memory stage h & 3; P_h aliases S[h & 3].
 //
 // Every wait is bounded; a wait that runs out raises a CTA-wide abort flag and the status word, the
 // roles drain, tensor memory is freed and the CTA exits.
@@ -32,30 +37,34 @@
 namespace heart {
 using namespace tc;
 
-constexpr int kAttnThreads = 320;
+constexpr int kAttnThreads = 352;
+constexpr int kStep = 64;   // keys per key step
+constexpr int kStages = 4;  // K / V ring depth = number of S buffers
 constexpr int kMaxNb = HEART_MAX_BLOCKS;
 
-// Shared-memory plan.  A key tile always holds 128 keys = SUBS key blocks of B tokens.
+// Shared-memory plan.
 template <int B>
 struct AttnSmem {
-  static constexpr int SUBS = 128 / B;          // key blocks per 128-key tile (1 or 2)
+  static constexpr int HPB = B / kStep;         // key steps per key block (1 or 2)
   static constexpr int QBT = 128 / B;           // query blocks per CTA (1 or 2)
-  static constexpr int TILE_BYTES = 128 * 256;  // [2 dim halves][128 rows][64] bf16, 128-byte swizzle
+  static constexpr int Q_BYTES = 128 * 256;     // [2 dim halves][128 rows][64] bf16, 128-byte swizzle
+  static constexpr int KV_BYTES = kStep * 256;  // [2 dim halves][64 rows][64] bf16, 128-byte swizzle
   static constexpr int OFF_Q = 0;
-  static constexpr int OFF_K = OFF_Q + TILE_BYTES;      // 2 stages: stream t uses stage t
-  static constexpr int OFF_V = OFF_K + 2 * TILE_BYTES;  // 2 stages
-  static constexpr int OFF_UNI = OFF_V + 2 * TILE_BYTES;  // int32[kMaxNb]: J | flags << 16
-  static constexpr int OFF_TBL = OFF_UNI + 4 * kMaxNb;    // uint32[kMaxNb]: flags per key block
-  static constexpr int OFF_XCH = OFF_TBL + 4 * kMaxNb;    // float[2 uses][2 streams][2 halves][128 rows]: row max, row sum
-  static constexpr int OFF_BAR = OFF_XCH + 4096;          // mbarriers and scalars
+  static constexpr int OFF_K = OFF_Q + Q_BYTES;
+  static constexpr int OFF_V = OFF_K + kStages * KV_BYTES;
+  static constexpr int OFF_UNI = OFF_V + kStages * KV_BYTES;  // int32[kMaxNb]: J | flags << 16
+  static constexpr int OFF_TBL = OFF_UNI + 4 * kMaxNb;        // uint32[kMaxNb]: flags per key block
+  static constexpr int OFF_XCH = OFF_TBL + 4 * kMaxNb;        // float[2 streams][2][128 rows]: max, sum
+  static constexpr int OFF_BAR = OFF_XCH + 2048;              // mbarriers and scalars
   static constexpr int TOTAL = OFF_BAR + 512;
 };
 
 struct AttnBars {
   uint64_t q_full;
-  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-  uint64_t s_full[2], p_full[2], pv_done[2];
-  uint64_t x_full[2][4];  // [stream][lane quarter]: the two column halves of the same 32 rows meet here
+  uint64_t k_full[kStages], v_full[kStages];  // TMA -> MMA issuer
+  uint64_t qk_done[kStages];                  // S_h complete: softmax may read it, K stage is free
+  uint64_t pv_done[kStages];                  // P_h V_h complete: V stage and S/P buffer are free
+  uint64_t p_full[kStages];                   // P_h written (one arrival per warp of the stream)
   uint32_t tmem_base;
   int n_union;
   int abort;
@@ -72,6 +81,20 @@ struct AttnParams {
   float scale_log2;
 };
 
+// Clock-stamp trace (compile with -DHEART_TRACE; the caller's lse buffer must then have one extra
+// row of N >= 4096 floats behind its R*N entries): CTA 0 records clock64() at the marked points of
+// its first 64 key steps.  Slots: 0-7 softmax warp 2, 16-23 softmax warp 6, 8-15 the MMA issuer.
+#ifdef HEART_TRACE
+#define HEART_TR(h, slot)                                                             \
+  do {                                                                                \
+    if (trace_base != nullptr && (h) < 64) trace_base[(h) * 32 + (slot)] = clock64(); \
+  } while (0)
+#else
+#define HEART_TR(h, slot) \
+  do {                    \
+  } while (0)
+#endif
+
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float r;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -83,7 +106,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
                    const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
   using L = AttnSmem<B>;
-  constexpr int SUBS = L::SUBS;
+  constexpr int HPB = L::HPB;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char *smem = reinterpret_cast<unsigned char *>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) &
                                                           ~static_cast<uintptr_t>(1023));
@@ -99,19 +122,21 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   const int bidx = r / p.H, hidx = r % p.H;
   const int row0 = cta_in_head * 128;  // first query token of this CTA
   const int nb = p.nb;
+#ifdef HEART_TRACE
+  long long *trace_base = (blockIdx.x == 0 && p.lse != nullptr)
+                              ? reinterpret_cast<long long *>(p.lse + (size_t)(gridDim.x / p.n_ctas_per_head) * p.N)
+                              : nullptr;
+#endif
 
   // ------------------------------------------------------------------ set-up
   if (tid == 0) {
     mbar_init(&bars->q_full, 1);
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&bars->s_full[i], 1);
-      mbar_init(&bars->p_full[i], 8);  // one arrival per softmax warp
-      for (int qq = 0; qq < 4; ++qq) mbar_init(&bars->x_full[i][qq], 2);
-      mbar_init(&bars->pv_done[i], 1);
+    for (int i = 0; i < kStages; ++i) {
       mbar_init(&bars->k_full[i], 1);
-      mbar_init(&bars->k_empty[i], 1);
       mbar_init(&bars->v_full[i], 1);
-      mbar_init(&bars->v_empty[i], 1);
+      mbar_init(&bars->qk_done[i], 1);
+      mbar_init(&bars->pv_done[i], 1);
+      mbar_init(&bars->p_full[i], 4);  // one arrival per warp of the stream's warpgroup
     }
     bars->abort = 0;
     bars->bad = 0;
@@ -165,165 +190,170 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
   const int U = bars->n_union;
-  const int NT = (U + SUBS - 1) / SUBS;  // 128-key tiles; tile k belongs to stream k & 1
+  const int NH = U * HPB;  // key steps; step h belongs to stream h & 1
+  // first key token of step h
+  auto key0_of = [&](int h) -> int { return (uni[h / HPB] & 0xffff) * B + (h % HPB) * kStep; };
 
   // ------------------------------------------------------------------ roles
-  if (warp < 2) {
-    if (warp == 0 && lane == 0) {  // ===== TMA producer
-      mbar_expect_tx(&bars->q_full, L::TILE_BYTES);
+  // Shared memory must not be released under a copy in flight: a producer that stops early (abort)
+  // waits, bounded, for the copies it has issued.
+  auto settle = [&](uint64_t *bar, uint32_t parity) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity) && clock64() - t0 < 40000000LL) {
+    }
+  };
+  if (warp == 0) {
+    if (lane == 0) {  // ===== TMA producer: Q once, then K_h into stage h & 3
+      mbar_expect_tx(&bars->q_full, L::Q_BYTES);
       tma_load_4d(Qs, &map_q, &bars->q_full, 0, row0, hidx, bidx);
       tma_load_4d(Qs + 128 * 128, &map_q, &bars->q_full, 64, row0, hidx, bidx);
-      int n_k = 0, n_v = 0;  // K and V tiles issued so far
-      for (int k = 0; k < NT; ++k) {
-        const int s = k & 1, ph = (k >> 1) & 1;
-        const int nsub = min(SUBS, U - k * SUBS);
-        if (k >= 2 && !mbar_wait(&bars->k_empty[s], ph ^ 1, abort)) break;
-        mbar_expect_tx(&bars->k_full[s], nsub * B * 256);
-        for (int sub = 0; sub < nsub; ++sub) {
-          const int J = uni[k * SUBS + sub] & 0xffff;
-          unsigned char *dst = Ks + s * L::TILE_BYTES + sub * (B * 128);
-          tma_load_4d(dst, &map_kv, &bars->k_full[s], 0, J * B, hidx, bidx);
-          tma_load_4d(dst + 128 * 128, &map_kv, &bars->k_full[s], 64, J * B, hidx, bidx);
-        }
-        n_k = k + 1;
-        if (k >= 2 && !mbar_wait(&bars->v_empty[s], ph ^ 1, abort)) break;
-        mbar_expect_tx(&bars->v_full[s], nsub * B * 256);
-        for (int sub = 0; sub < nsub; ++sub) {
-          const int J = uni[k * SUBS + sub] & 0xffff;
-          unsigned char *dst = Vs + s * L::TILE_BYTES + sub * (B * 128);
-          tma_load_4d(dst, &map_v, &bars->v_full[s], 0, J * B, hidx, bidx);
-          tma_load_4d(dst + 128 * 128, &map_v, &bars->v_full[s], 64, J * B, hidx, bidx);
-        }
-        n_v = k + 1;
+      int issued = 0;
+      for (int h = 0; h < NH; ++h) {
+        const int s = h & 3, ph = (h >> 2) & 1;
+        // the stage is free once S_{h-4} = Q K_{h-4}^T is complete
+        if (h >= kStages && !mbar_wait(&bars->qk_done[s], ph ^ 1, abort)) break;
+        const int key0 = key0_of(h);
+        unsigned char *dst = Ks + s * L::KV_BYTES;
+        mbar_expect_tx(&bars->k_full[s], L::KV_BYTES);
+        tma_load_4d(dst, &map_kv, &bars->k_full[s], 0, key0, hidx, bidx);
+        tma_load_4d(dst + kStep * 128, &map_kv, &bars->k_full[s], 64, key0, hidx, bidx);
+        issued = h + 1;
       }
-      // Shared memory must not be released under a copy in flight: the Q tile is always awaited here
-      // (nobody else does when the union is empty), and after an abort so are the last K/V copies.
-      auto settle = [&](uint64_t *bar, uint32_t parity) {
-        const long long t0 = clock64();
-        while (!mbar_try_wait(bar, parity) && clock64() - t0 < 40000000LL) {
-        }
-      };
-      settle(&bars->q_full, 0);
-      if (*abort) {
-        for (int k = (n_k > 2 ? n_k - 2 : 0); k < n_k; ++k) settle(&bars->k_full[k & 1], (k >> 1) & 1);
-        for (int k = (n_v > 2 ? n_v - 2 : 0); k < n_v; ++k) settle(&bars->v_full[k & 1], (k >> 1) & 1);
+      settle(&bars->q_full, 0);  // nobody else waits for Q when the union is empty
+      if (*abort)
+        for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->k_full[h & 3], (h >> 2) & 1);
+    }
+  } else if (warp == 10) {
+    if (lane == 0) {  // ===== TMA producer: V_h into stage h & 3
+      int issued = 0;
+      for (int h = 0; h < NH; ++h) {
+        const int s = h & 3, ph = (h >> 2) & 1;
+        if (h >= kStages && !mbar_wait(&bars->pv_done[s], ph ^ 1, abort)) break;
+        const int key0 = key0_of(h);
+        unsigned char *dst = Vs + s * L::KV_BYTES;
+        mbar_expect_tx(&bars->v_full[s], L::KV_BYTES);
+        tma_load_4d(dst, &map_v, &bars->v_full[s], 0, key0, hidx, bidx);
+        tma_load_4d(dst + kStep * 128, &map_v, &bars->v_full[s], 64, key0, hidx, bidx);
+        issued = h + 1;
       }
-    } else if (warp == 1 && lane == 0 && NT > 0) {  // ===== MMA issuer
-      constexpr uint32_t idesc_qk_full = idesc_bf16_f32(128, 128, false, false);
-      constexpr uint32_t idesc_qk_half = idesc_bf16_f32(128, 64, false, false);
+      if (*abort)
+        for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->v_full[h & 3], (h >> 2) & 1);
+    }
+  } else if (warp == 1) {
+    if (NH > 0) {  // ===== MMA issuer: the whole warp runs the loop (uniform control flow keeps the
+                   // descriptors in uniform registers), one elected lane issues
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(128, kStep, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, 128, false, true);
-      // descriptors differ only in the 14-bit start-address field: base + constant per k-step
+      // Descriptors of one key step differ only in the start-address field (low word, no carry out
+      // of it): base + a compile-time offset per 16-element k-step.
+      //   Q, K (K-major): 64 dims = one 128-byte row; dim halves Q: 128*128 B apart, K: 64*128 B.
+      //   V (MN-major):   64 dims = one 128-byte row; dim halves 64*128 B apart (the LBO);
+      //                   16 keys = 16 rows = 2048 B per k-step.
       const uint64_t q_desc = smem_desc_sw128(smem_u32(Qs), 16, 1024);
       const uint64_t k_desc = smem_desc_sw128(smem_u32(Ks), 16, 1024);
-      const uint64_t v_desc = smem_desc_sw128(smem_u32(Vs), 128 * 128, 1024);
-      bool ok = true;
-      auto keys_in = [&](int k) -> int { return min(SUBS, U - k * SUBS) * B; };
-      // every descriptor is formed once, outside the loop: issuing a tile is 8 back-to-back MMAs
-      uint64_t qd[8], kd[2][8], vd[2][8];
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        qd[ks] = q_desc + ((ks >> 2) * 1024 + (ks & 3) * 2);
-        kd[0][ks] = k_desc + ((ks >> 2) * 1024 + (ks & 3) * 2);
-        kd[1][ks] = kd[0][ks] + (L::TILE_BYTES >> 4);
-        vd[0][ks] = v_desc + ks * 128;
-        vd[1][ks] = vd[0][ks] + (L::TILE_BYTES >> 4);
-      }
-      auto issue_qk = [&](int k) {  // S_t = Q K_k^T, t = k & 1; K_k sits in stage t
-        const int t = k & 1;
-        const uint32_t d = tmem + t * 128;
-        const uint32_t idesc = keys_in(k) == 128 ? idesc_qk_full : idesc_qk_half;
-        if (t == 0) {
-          mma_ss(d, qd[0], kd[0][0], idesc, 0u);
-#pragma unroll
-          for (int ks = 1; ks < 8; ++ks) mma_ss(d, qd[ks], kd[0][ks], idesc, 1u);
-        } else {
-          mma_ss(d, qd[0], kd[1][0], idesc, 0u);
-#pragma unroll
-          for (int ks = 1; ks < 8; ++ks) mma_ss(d, qd[ks], kd[1][ks], idesc, 1u);
-        }
-        tc_commit(&bars->s_full[t]);
-        tc_commit(&bars->k_empty[t]);
+      const uint64_t v_desc = smem_desc_sw128(smem_u32(Vs), kStep * 128, 1024);
+      auto at = [](uint64_t desc, uint32_t off16) -> uint64_t {
+        return (desc & 0xffffffff00000000ull) | (uint32_t)((uint32_t)desc + off16);
       };
-      auto issue_pv = [&](int k) {  // O_t (+)= P_t V_k
-        const int t = k & 1;
-        const uint32_t d = tmem + 256 + t * 128, pa = tmem + t * 128;
-        const int ksteps = keys_in(k) / 16;
-        if (t == 0) {
-          mma_ts(d, pa, vd[0][0], idesc_pv, k >= 2 ? 1u : 0u);
+      const bool leader = elect_one();  // the same lane every time: commits track its MMAs
+      auto issue_qk = [&](int h) {  // S[h & 3] = Q K_h^T
+        const int s = h & 3;
+        const uint32_t d = tmem + 256 + s * kStep;
+        const uint64_t ks_desc = at(k_desc, s * (L::KV_BYTES >> 4));
+        if (leader) {
 #pragma unroll
-          for (int ks = 1; ks < 8; ++ks)
-            if (ks < ksteps) mma_ts(d, pa + ks * 8, vd[0][ks], idesc_pv, 1u);
-        } else {
-          mma_ts(d, pa, vd[1][0], idesc_pv, k >= 2 ? 1u : 0u);
-#pragma unroll
-          for (int ks = 1; ks < 8; ++ks)
-            if (ks < ksteps) mma_ts(d, pa + ks * 8, vd[1][ks], idesc_pv, 1u);
+          for (int ks = 0; ks < 8; ++ks)
+            mma_ss(d, at(q_desc, (ks >> 2) * 1024 + (ks & 3) * 2), at(ks_desc, (ks >> 2) * 512 + (ks & 3) * 2), idesc_qk,
+                   ks > 0 ? 1u : 0u);
+          tc_commit(&bars->qk_done[s]);
         }
-        tc_commit(&bars->pv_done[t]);
-        tc_commit(&bars->v_empty[t]);
+        __syncwarp();
       };
-      ok = mbar_wait(&bars->q_full, 0, abort);
-      for (int k = 0; k < 2 && k < NT && ok; ++k) {
-        ok = mbar_wait(&bars->k_full[k], 0, abort);
+      auto issue_pv = [&](int h) {  // O_t (+)= P_h V_h, t = h & 1; P_h sits over S[h & 3]
+        const int s = h & 3;
+        const uint32_t d = tmem + (h & 1) * 128, pa = tmem + 256 + s * kStep;
+        const uint64_t vs_desc = at(v_desc, s * (L::KV_BYTES >> 4));
+        if (leader) {
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) mma_ts(d, pa + ks * 8, at(vs_desc, ks * 128), idesc_pv, (h >= 2 || ks > 0) ? 1u : 0u);
+          tc_commit(&bars->pv_done[s]);
+        }
+        __syncwarp();
+      };
+      bool ok = mbar_wait(&bars->q_full, 0, abort);
+      for (int h = 0; h < kStages && h < NH && ok; ++h) {
+        ok = mbar_wait(&bars->k_full[h], 0, abort);
         if (ok) {
           tc_fence_after();
-          issue_qk(k);
+          issue_qk(h);
         }
       }
-      for (int k = 0; k < NT && ok; ++k) {
-        const int t = k & 1, ph = (k >> 1) & 1;
-        ok = mbar_wait(&bars->v_full[t], ph, abort);
-        if (ok) ok = mbar_wait(&bars->p_full[t], ph, abort);
+      for (int h = 0; h < NH && ok; ++h) {
+        const int s = h & 3, ph = (h >> 2) & 1;
+        ok = mbar_wait(&bars->v_full[s], ph, abort);
+        HEART_TR(h, 12);
+        if (ok) ok = mbar_wait(&bars->p_full[s], ph, abort);
         if (!ok) break;
+        HEART_TR(h, 8);
         tc_fence_after();
-        issue_pv(k);
-        if (k + 2 < NT) {
-          ok = mbar_wait(&bars->k_full[t], ph ^ 1, abort);
+        issue_pv(h);
+        HEART_TR(h, 9);
+        if (h + kStages < NH) {  // S[s] is free again once P_h V_h has read it: same pipe, in order
+          ok = mbar_wait(&bars->k_full[s], ph ^ 1, abort);
           if (!ok) break;
+          HEART_TR(h, 10);
           tc_fence_after();
-          issue_qk(k + 2);
+          issue_qk(h + kStages);
+          HEART_TR(h, 11);
         }
       }
     }
   } else {
-    // ===== softmax / correction / epilogue: thread = (query row, half of the key columns), both streams
-    // The stream index t is a run-time value on purpose: one compact copy of this code serves both
-    // streams, which keeps the loop inside the instruction cache.
-    const int a = (warp - 2) >> 2;  // column half: S columns [64a, 64a+64), O columns [64a, 64a+64)
+    // ===== softmax / correction / epilogue: warpgroup t owns stream t, thread = one query row
+    // The stream index t is a run-time value (uniform per warp): both warpgroups run one copy of
+    // this code.
+    const int t = (warp - 2) >> 2;  // stream of this warpgroup; it processes key steps h = t, t+2, ...
     const int q = warp & 3;         // TMEM lane quarter this warp may touch
     const int row = q * 32 + lane;  // row inside the 128-row query tile
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+    const uint32_t o_addr = lane_addr + t * 128;
     const float c = p.scale_log2;
-    float m_ref0 = -INFINITY, m_ref1 = -INFINITY, l_part0 = 0.f, l_part1 = 0.f;
+    float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
-    const int my_sub = (a * 64) / B;             // key sub-block this thread's columns belong to
-    const int col_in_sub = a * 64 - my_sub * B;  // first of its columns inside that sub-block
-    const uint32_t my_bit = 1u << (row / B);     // query block of this row (uniform within a warp)
-    for (int k = 0; k < NT && ok; ++k) {
-      const int t = k & 1, n_act = k >> 1;
-      const int nsub = min(SUBS, U - k * SUBS);
-      // valid key columns, for this row, of the thread's two 32-column chunks
-      int lim0 = 0, lim1 = 0;
-      if (my_sub < nsub) {
-        const uint32_t e = (uint32_t)uni[k * SUBS + my_sub];
-        if ((e >> 16) & my_bit) {
-          const int v = min(B, p.N - (int)(e & 0xffff) * B) - col_in_sub;
-          lim0 = max(0, min(32, v));
-          lim1 = max(0, min(32, v - 32));
-        }
+    const uint32_t my_bit = 1u << (row / B);  // query block of this row (uniform within a warp)
+#ifdef HEART_TRACE
+    const int tr0 = t ? 16 : 0;
+    const bool trw = (warp == 2 || warp == 6) && lane == 0;
+#define HEART_TRS(slot)                   \
+  do {                                    \
+    if (trw) HEART_TR(h, tr0 + (slot));   \
+  } while (0)
+#else
+#define HEART_TRS(slot) \
+  do {                  \
+  } while (0)
+#endif
+    for (int h = t; h < NH && ok; h += 2) {
+      const int s = h & 3, ph = (h >> 2) & 1;
+      HEART_TRS(0);
+      // key columns of this step that are real keys this row attends to
+      int lim = 0;
+      {
+        const uint32_t e = (uint32_t)uni[h / HPB];
+        if ((e >> 16) & my_bit) lim = max(0, min(kStep, p.N - ((int)(e & 0xffff) * B + (h % HPB) * kStep)));
       }
-      float m_ref = t ? m_ref1 : m_ref0;
-      const uint32_t s_addr = lane_addr + t * 128 + a * 64;
-      const uint32_t o_addr = lane_addr + 256 + t * 128 + a * 64;
-      float *xrow = xch + (t * 2) * 128 + row;  // [t][half][row]
-      ok = __all_sync(0xffffffffu, mbar_wait(&bars->s_full[t], n_act & 1, abort));
+      const int lim0 = min(lim, 32), lim1 = max(lim - 32, 0);
+      const uint32_t s_addr = lane_addr + 256 + s * kStep;
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->qk_done[s], ph, abort));
       if (!ok) break;
+      HEART_TRS(1);
       tc_fence_after();
       uint32_t sreg[64];
       if (lim0 > 0) tmem_ld32(s_addr, *reinterpret_cast<uint32_t(*)[32]>(&sreg[0]));
       if (lim1 > 0) tmem_ld32(s_addr + 32, *reinterpret_cast<uint32_t(*)[32]>(&sreg[32]));
       tmem_wait_ld();
-      if (lim0 < 32 || lim1 < 32) {  // rare: ragged last block or a sub-block this row does not list
+      HEART_TRS(2);
+      if (lim < kStep) {  // rare: ragged last block, or a block this row's query block does not list
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           if (i >= lim0) sreg[i] = 0xff800000u;  // -inf: ignored by the max, 2^-inf = 0
@@ -338,14 +368,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         mx2 = fmax3(mx2, __uint_as_float(sreg[i + 4]), __uint_as_float(sreg[i + 5]));
         mx3 = fmax3(mx3, __uint_as_float(sreg[i + 6]), __uint_as_float(sreg[i + 7]));
       }
-      // the two column halves of a row exchange their maxima
-      const float mx_mine = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      xrow[a * 128] = mx_mine;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->x_full[t][q]);
-      ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[t][q], n_act & 1, abort));
-      if (!ok) break;
-      const float x_max = fmaxf(mx_mine, xrow[(1 - a) * 128]) * c;  // -inf stays -inf (c > 0)
+      const float x_max = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c;  // -inf stays -inf (c > 0)
+      HEART_TRS(3);
       float alpha = 1.f;
       bool grow = false;
       if (m_ref == -INFINITY) {
@@ -355,97 +379,94 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         m_ref = x_max;
         grow = true;
       }
-      if (__any_sync(0xffffffffu, grow) && n_act > 0) {
-        // O_t must be quiescent: the latest PV of this stream has to be complete
-        ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[t], (n_act - 1) & 1, abort));
+      if (__any_sync(0xffffffffu, grow) && h >= 2) {
+        // O_t must be quiescent: the previous product of this stream has to be complete
+        ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(h - 2) & 3], ((h - 2) >> 2) & 1, abort));
         if (!ok) break;
         tc_fence_after();
+        const uint64_t alpha2 = pack_f32x2(alpha, alpha);
 #pragma unroll 1
-        for (int ch = 0; ch < 2; ++ch) {
+        for (int ch = 0; ch < 4; ++ch) {
           uint32_t v[32];
           tmem_ld32(o_addr + ch * 32, v);
           tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+          for (int i = 0; i < 32; i += 2) {
+            float lo, hi;
+            unpack_f32x2(mul_f32x2(pack_f32x2(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), alpha2), lo, hi);
+            v[i] = __float_as_uint(lo);
+            v[i + 1] = __float_as_uint(hi);
+          }
           tmem_st32(o_addr + ch * 32, v);
         }
         tmem_wait_st();
       }
+      HEART_TRS(4);
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      // p = 2^(s*c - m), packed to bf16 over columns [32a, 32a+32) of S_t
-      float sum0 = 0.f, sum1 = 0.f;
-      if (a * 64 < nsub * B) {  // else: sub-block absent from this tile, the PV product skips its keys
+      const uint64_t c2 = pack_f32x2(c, c), neg_m2 = pack_f32x2(neg_m, neg_m);
+      // p = 2^(s*c - m), packed to bf16 over columns [0, 32) of S[h & 3]; the product reads all 64
+      // keys of the step, so every column is written (zeros where the row has no key)
+      float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          uint32_t pk[16];
-          if ((ch ? lim1 : lim0) == 0) {  // this row lists nothing here: zeros, no exponentials
+      for (int ch = 0; ch < 2; ++ch) {
+        uint32_t pk[16];
+        if ((ch ? lim1 : lim0) == 0) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) pk[i] = 0u;
-          } else
+          for (int i = 0; i < 16; ++i) pk[i] = 0u;
+        } else {
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            const float p0 = ex2(fmaf(__uint_as_float(sreg[ch * 32 + i]), c, neg_m));
-            const float p1 = ex2(fmaf(__uint_as_float(sreg[ch * 32 + i + 1]), c, neg_m));
+          for (int i = 0; i < 32; i += 4) {
+            float x0, x1, x2, x3;
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sreg[ch * 32 + i]), __uint_as_float(sreg[ch * 32 + i + 1])), c2, neg_m2), x0, x1);
+            unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sreg[ch * 32 + i + 2]), __uint_as_float(sreg[ch * 32 + i + 3])), c2, neg_m2), x2, x3);
             // the row sum is taken over the bf16-rounded weights, the ones the PV product really
             // uses, so numerator and denominator carry the same rounding: O stays a weighted mean
-            const uint32_t w = pack_bf16x2(p0, p1);
-            pk[i >> 1] = w;
-            sum0 += __uint_as_float(w << 16);
-            sum1 += __uint_as_float(w & 0xffff0000u);
+            const uint32_t w0 = pack_bf16x2(ex2(x0), ex2(x1));
+            const uint32_t w1 = pack_bf16x2(ex2(x2), ex2(x3));
+            pk[i >> 1] = w0;
+            pk[(i >> 1) + 1] = w1;
+            add_bf16x2_to_f32(sum0, sum1, w0);
+            add_bf16x2_to_f32(sum2, sum3, w1);
           }
-          tmem_st16(lane_addr + t * 128 + a * 32 + ch * 16, pk);
         }
+        tmem_st16(s_addr + ch * 16, pk);
       }
-      const float l_new = (t ? l_part1 : l_part0) * alpha + (sum0 + sum1);
+      l_run = l_run * alpha + ((sum0 + sum1) + (sum2 + sum3));
+      HEART_TRS(5);
       tmem_wait_st();
+      HEART_TRS(6);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->p_full[t]);
-      if (t) {
-        m_ref1 = m_ref;
-        l_part1 = l_new;
-      } else {
-        m_ref0 = m_ref;
-        l_part0 = l_new;
-      }
+      if (lane == 0) mbar_arrive(&bars->p_full[s]);
+      HEART_TRS(7);
     }
-    // epilogue: merge the two streams; each warpgroup writes its 64-dim half of the output rows
-    const int n0 = (NT + 1) >> 1, n1 = NT >> 1;  // tiles per stream
+    // epilogue: the two warpgroups exchange (max, sum) of their streams; warpgroup t then writes
+    // output dims [64t, 64t+64) of every row from both accumulators
+    const int n0 = (NH + 1) >> 1, n1 = NH >> 1;  // key steps per stream
     const int tok = row0 + row;
     const bool valid_row = tok < p.N;
-    float l0 = l_part0, l1 = l_part1;
-    if (ok && n0 > 0) {  // the column halves add their partial row sums (stream 0, then stream 1)
-      // (own slots, not the ones of the row maxima: a slow partner may still be reading those)
-      xch[512 + row + a * 128] = l_part0;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->x_full[0][q]);
-      ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[0][q], n0 & 1, abort));
-      if (ok) l0 += xch[512 + row + (1 - a) * 128];
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[0], (n0 - 1) & 1, abort));
-    }
-    if (ok && n1 > 0) {
-      xch[768 + row + a * 128] = l_part1;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars->x_full[1][q]);
-      ok = __all_sync(0xffffffffu, mbar_wait(&bars->x_full[1][q], n1 & 1, abort));
-      if (ok) l1 += xch[768 + row + (1 - a) * 128];
-      if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[1], (n1 - 1) & 1, abort));
-    }
+    xch[t * 256 + row] = m_ref;
+    xch[t * 256 + 128 + row] = l_run;
+    asm volatile("bar.sync 1, 256;" ::: "memory");  // the eight softmax warps (every one gets here)
+    ok = ok && !*abort;
+    const float m0 = xch[row], l0 = xch[128 + row], m1 = xch[256 + row], l1 = xch[384 + row];
+    // the products complete in issue order: the last one covers both streams
+    if (ok && NH > 0) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(NH - 1) & 3], ((NH - 1) >> 2) & 1, abort));
     if (ok) {
       tc_fence_after();
-      const float m = fmaxf(m_ref0, m_ref1);
-      const float w0 = (n0 > 0 && m_ref0 > -INFINITY) ? ex2(m_ref0 - m) : 0.f;
-      const float w1 = (n1 > 0 && m_ref1 > -INFINITY) ? ex2(m_ref1 - m) : 0.f;
+      const float m = fmaxf(m0, m1);
+      const float w0 = (n0 > 0 && m0 > -INFINITY) ? ex2(m0 - m) : 0.f;
+      const float w1 = (n1 > 0 && m1 > -INFINITY) ? ex2(m1 - m) : 0.f;
       const float l = l0 * w0 + l1 * w1;
       const float inv = l > 0.f ? 1.f / l : 0.f;
       const float f0 = w0 * inv, f1 = w1 * inv;
-      uint16_t *orow = p.O + (long long)bidx * p.sb + (long long)hidx * p.sh + (long long)tok * p.sn + a * 64;
-      const uint32_t o_addr = lane_addr + 256 + a * 64;
+      uint16_t *orow = p.O + (long long)bidx * p.sb + (long long)hidx * p.sh + (long long)tok * p.sn + t * 64;
+      const uint32_t o_base = lane_addr + t * 64;
 #pragma unroll 1
       for (int ch = 0; ch < 4; ++ch) {  // 16 output dims at a time
         uint32_t v0[16], v1[16];
-        if (n0 > 0) tmem_ld16(o_addr + ch * 16, v0);
-        if (n1 > 0) tmem_ld16(o_addr + 128 + ch * 16, v1);
+        if (n0 > 0) tmem_ld16(o_base + ch * 16, v0);
+        if (n1 > 0) tmem_ld16(o_base + 128 + ch * 16, v1);
         tmem_wait_ld();
         float o[16];
 #pragma unroll
@@ -466,7 +487,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
           }
         }
       }
-      if (a == 0 && valid_row && p.lse != nullptr)
+      if (t == 0 && valid_row && p.lse != nullptr)
         p.lse[(size_t)r * p.N + tok] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
@@ -530,7 +551,7 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,
                              float *lse, int32_t *status, cudaStream_t s, int *launches) {
   CUtensorMap mq, mk, mv;
-  if (!make_map(&mq, Q, g, 128) || !make_map(&mk, K, g, g.block) || !make_map(&mv, V, g, g.block))
+  if (!make_map(&mq, Q, g, 128) || !make_map(&mk, K, g, kStep) || !make_map(&mv, V, g, kStep))
     return cudaErrorInvalidValue;
   AttnParams prm;
   prm.kv_idx = kv_idx;
