@@ -13,17 +13,18 @@
 // in tensor memory: S of the stream's next step is computed while the softmax works on the current
 // one, so the serial chain softmax -> P V -> Q K^T -> softmax is off the critical path.
 //
-// Warp roles (352 threads):
-//   warp 0      TMA producer for Q (once) and K, through a four-stage shared-memory ring
-//               (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers).
-//   warp 1      MMA issuer (one lane): S_h = Q K_h^T into tensor memory (tcgen05.mma, operands in
-//               shared memory) and O_t += P_h V_h with P_h read from tensor memory.
-//   warps 2-5   softmax warpgroup of stream 0; warps 6-9 of stream 1.  Per key step a thread reads
+// Warp roles (512 threads; registers are moved from the helper warps to the softmax warps at start):
+//   warps 0-3   softmax warpgroup of stream 0; warps 4-7 of stream 1.  Per key step a thread reads
 //               its row of S (64 columns), takes the max, rescales its row of O only when the max
 //               grew by more than 2^8, writes P = 2^(s*scale*log2e - m) as bf16 over the first half
 //               of the S buffer and adds the row sum.  At the end the two warpgroups exchange
 //               (max, sum), and warpgroup t writes output dims [64t, 64t+64) of every row (and lse).
-//   warp 10     TMA producer for V (its own ring: V_h is needed four key steps later than K_h).
+//   warp 8      TMA producer for Q (once) and K, through a four-stage shared-memory ring
+//               (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers).
+//   warp 9      TMA producer for V (its own ring: V_h is needed four key steps later than K_h).
+//   warp 10     MMA issuer (one elected lane) of O_t += P_h V_h, P_h read from tensor memory.
+//   warps 12-15 MMA issuers of S_h = Q K_h^T (tcgen05.mma, operands in shared memory), warp 12+i
+//               for the key steps h = i (mod 4).
 // Tensor memory (512 columns): O_0 | O_1 | S[4]  =  128 + 128 + 4 x 64; key step h uses S[h & 3]
 // (stream h & 1, buffer (h >> 1) & 1) and shared-memory stage h & 3; P_h aliases S[h & 3].
 //
@@ -37,7 +38,11 @@
 namespace heart {
 using namespace tc;
 
-constexpr int kAttnThreads = 352;
+constexpr int kAttnThreads = 512;
+// warp roles: 0-3 softmax of stream 0, 4-7 softmax of stream 1 (lane quarter = warp & 3), then the
+// helpers, two per SM sub-partition (warp & 3)
+constexpr int kWarpKProd = 8, kWarpVProd = 9, kWarpPV = 10, kWarpQK0 = 12;  // QK issuers: 12..15
+constexpr int kRegsSoftmax = 176, kRegsHelper = 80;  // 2 * (176 + 80) * 32 lanes = one sub-partition
 constexpr int kStep = 64;   // keys per key step
 constexpr int kStages = 4;  // K / V ring depth = number of S buffers
 constexpr int kMaxNb = HEART_MAX_BLOCKS;
@@ -163,12 +168,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         atomicOr(&tbl[J], 1u << qb);
     }
   }
-  if (warp == 1) {
+  if (warp == kWarpQK0) {
     tmem_alloc(&bars->tmem_base, 512);
     tmem_relinquish();
   }
   __syncthreads();
-  if (warp == 0) {  // ascending compaction of the flagged key blocks
+  if (warp == kWarpKProd) {  // ascending compaction of the flagged key blocks
     int count = 0;
     for (int base = 0; base < nb; base += 32) {
       const int J = base + lane;
@@ -202,7 +207,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     while (!mbar_try_wait(bar, parity) && clock64() - t0 < 40000000LL) {
     }
   };
-  if (warp == 0) {
+  if (warp >= 8) setmaxnreg_dec<kRegsHelper>();
+  if (warp == kWarpKProd) {
     if (lane == 0) {  // ===== TMA producer: Q once, then K_h into stage h & 3
       mbar_expect_tx(&bars->q_full, L::Q_BYTES);
       tma_load_4d(Qs, &map_q, &bars->q_full, 0, row0, hidx, bidx);
@@ -211,7 +217,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       for (int h = 0; h < NH; ++h) {
         const int s = h & 3, ph = (h >> 2) & 1;
         // the stage is free once S_{h-4} = Q K_{h-4}^T is complete
-        if (h >= kStages && !mbar_wait(&bars->qk_done[s], ph ^ 1, abort)) break;
+        if (h >= kStages && !mbar_wait_relaxed(&bars->qk_done[s], ph ^ 1, abort)) break;
         const int key0 = key0_of(h);
         unsigned char *dst = Ks + s * L::KV_BYTES;
         mbar_expect_tx(&bars->k_full[s], L::KV_BYTES);
@@ -223,12 +229,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       if (*abort)
         for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->k_full[h & 3], (h >> 2) & 1);
     }
-  } else if (warp == 10) {
+  } else if (warp == kWarpVProd) {
     if (lane == 0) {  // ===== TMA producer: V_h into stage h & 3
       int issued = 0;
       for (int h = 0; h < NH; ++h) {
         const int s = h & 3, ph = (h >> 2) & 1;
-        if (h >= kStages && !mbar_wait(&bars->pv_done[s], ph ^ 1, abort)) break;
+        if (h >= kStages && !mbar_wait_relaxed(&bars->pv_done[s], ph ^ 1, abort)) break;
         const int key0 = key0_of(h);
         unsigned char *dst = Vs + s * L::KV_BYTES;
         mbar_expect_tx(&bars->v_full[s], L::KV_BYTES);
@@ -239,9 +245,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       if (*abort)
         for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->v_full[h & 3], (h >> 2) & 1);
     }
-  } else if (warp == 1) {
-    if (NH > 0) {  // ===== MMA issuer: the whole warp runs the loop (uniform control flow keeps the
-                   // descriptors in uniform registers), one elected lane issues
+  } else if (warp == kWarpPV || warp >= kWarpQK0) {
+    // ===== MMA issuers.  Warp 12+i issues S_h = Q K_h^T for the key steps h = i, i+4, ... (buffer
+    // and stage i); warp 10 issues every O_t += P_h V_h.  An MMA that waits for the tensor pipe
+    // holds up the other warps of its SM sub-partition, so the S products -- eight MMAs per key
+    // step -- rotate over the four sub-partitions.  The whole warp runs the loop (uniform control
+    // flow keeps the descriptors in uniform registers), one elected lane issues.
+    if (NH > 0) {
       constexpr uint32_t idesc_qk = idesc_bf16_f32(128, kStep, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, 128, false, true);
       // Descriptors of one key step differ only in the start-address field (low word, no carry out
@@ -249,70 +259,76 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       //   Q, K (K-major): 64 dims = one 128-byte row; dim halves Q: 128*128 B apart, K: 64*128 B.
       //   V (MN-major):   64 dims = one 128-byte row; dim halves 64*128 B apart (the LBO);
       //                   16 keys = 16 rows = 2048 B per k-step.
-      const uint64_t q_desc = smem_desc_sw128(smem_u32(Qs), 16, 1024);
-      const uint64_t k_desc = smem_desc_sw128(smem_u32(Ks), 16, 1024);
-      const uint64_t v_desc = smem_desc_sw128(smem_u32(Vs), kStep * 128, 1024);
       auto at = [](uint64_t desc, uint32_t off16) -> uint64_t {
         return (desc & 0xffffffff00000000ull) | (uint32_t)((uint32_t)desc + off16);
       };
       const bool leader = elect_one();  // the same lane every time: commits track its MMAs
-      auto issue_qk = [&](int h) {  // S[h & 3] = Q K_h^T
-        const int s = h & 3;
+      bool ok = true;
+      if (warp >= kWarpQK0) {
+        const int s = warp - kWarpQK0;  // S buffer and K stage of this warp
+        const uint64_t q_desc = smem_desc_sw128(smem_u32(Qs), 16, 1024);
+        const uint64_t k_desc = smem_desc_sw128(smem_u32(Ks) + s * L::KV_BYTES, 16, 1024);
         const uint32_t d = tmem + 256 + s * kStep;
-        const uint64_t ks_desc = at(k_desc, s * (L::KV_BYTES >> 4));
-        if (leader) {
+        auto issue_qk = [&]() {  // S[s] = Q K^T with the K tile that sits in stage s
+          if (leader) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks)
-            mma_ss(d, at(q_desc, (ks >> 2) * 1024 + (ks & 3) * 2), at(ks_desc, (ks >> 2) * 512 + (ks & 3) * 2), idesc_qk,
-                   ks > 0 ? 1u : 0u);
-          tc_commit(&bars->qk_done[s]);
+            for (int ks = 0; ks < 8; ++ks)
+              mma_ss(d, at(q_desc, (ks >> 2) * 1024 + (ks & 3) * 2), at(k_desc, (ks >> 2) * 512 + (ks & 3) * 2), idesc_qk,
+                     ks > 0 ? 1u : 0u);
+            tc_commit(&bars->qk_done[s]);
+          }
+          __syncwarp();
+        };
+        if (s < NH) {
+          ok = mbar_wait(&bars->q_full, 0, abort);
+          if (ok) ok = mbar_wait(&bars->k_full[s], 0, abort);
+          if (ok) {
+            tc_fence_after();
+            issue_qk();
+          }
         }
-        __syncwarp();
-      };
-      auto issue_pv = [&](int h) {  // O_t (+)= P_h V_h, t = h & 1; P_h sits over S[h & 3]
-        const int s = h & 3;
-        const uint32_t d = tmem + (h & 1) * 128, pa = tmem + 256 + s * kStep;
-        const uint64_t vs_desc = at(v_desc, s * (L::KV_BYTES >> 4));
-        if (leader) {
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks) mma_ts(d, pa + ks * 8, at(vs_desc, ks * 128), idesc_pv, (h >= 2 || ks > 0) ? 1u : 0u);
-          tc_commit(&bars->pv_done[s]);
-        }
-        __syncwarp();
-      };
-      bool ok = mbar_wait(&bars->q_full, 0, abort);
-      for (int h = 0; h < kStages && h < NH && ok; ++h) {
-        ok = mbar_wait(&bars->k_full[h], 0, abort);
-        if (ok) {
-          tc_fence_after();
-          issue_qk(h);
-        }
-      }
-      for (int h = 0; h < NH && ok; ++h) {
-        const int s = h & 3, ph = (h >> 2) & 1;
-        ok = mbar_wait(&bars->v_full[s], ph, abort);
-        HEART_TR(h, 12);
-        if (ok) ok = mbar_wait(&bars->p_full[s], ph, abort);
-        if (!ok) break;
-        HEART_TR(h, 8);
-        tc_fence_after();
-        issue_pv(h);
-        HEART_TR(h, 9);
-        if (h + kStages < NH) {  // S[s] is free again once P_h V_h has read it: same pipe, in order
+        for (int h = s; h + kStages < NH && ok; h += kStages) {
+          const int ph = (h >> 2) & 1;
+          // S[s] holds P_h until the product P_h V_h has read it
           ok = mbar_wait(&bars->k_full[s], ph ^ 1, abort);
+          if (ok) ok = mbar_wait(&bars->pv_done[s], ph, abort);
           if (!ok) break;
           HEART_TR(h, 10);
           tc_fence_after();
-          issue_qk(h + kStages);
+          issue_qk();
           HEART_TR(h, 11);
+        }
+      } else {
+        const uint64_t v_desc = smem_desc_sw128(smem_u32(Vs), kStep * 128, 1024);
+        for (int h = 0; h < NH && ok; ++h) {  // O_t (+)= P_h V_h, t = h & 1; P_h sits over S[h & 3]
+          const int s = h & 3, ph = (h >> 2) & 1;
+          ok = mbar_wait(&bars->v_full[s], ph, abort);
+          HEART_TR(h, 12);
+          if (ok) ok = mbar_wait(&bars->p_full[s], ph, abort);
+          if (!ok) break;
+          HEART_TR(h, 8);
+          tc_fence_after();
+          const uint32_t d = tmem + (h & 1) * 128, pa = tmem + 256 + s * kStep;
+          const uint64_t vs_desc = at(v_desc, s * (L::KV_BYTES >> 4));
+          if (leader) {
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks)
+              mma_ts(d, pa + ks * 8, at(vs_desc, ks * 128), idesc_pv, (h >= 2 || ks > 0) ? 1u : 0u);
+            tc_commit(&bars->pv_done[s]);
+          }
+          __syncwarp();
+          HEART_TR(h, 9);
         }
       }
     }
+  } else if (warp >= 8) {
+    // warp 11: no role (it completes the helper warpgroups)
   } else {
     // ===== softmax / correction / epilogue: warpgroup t owns stream t, thread = one query row
     // The stream index t is a run-time value (uniform per warp): both warpgroups run one copy of
     // this code.
-    const int t = (warp - 2) >> 2;  // stream of this warpgroup; it processes key steps h = t, t+2, ...
+    setmaxnreg_inc<kRegsSoftmax>();
+    const int t = warp >> 2;        // stream of this warpgroup; it processes key steps h = t, t+2, ...
     const int q = warp & 3;         // TMEM lane quarter this warp may touch
     const int row = q * 32 + lane;  // row inside the 128-row query tile
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
@@ -323,7 +339,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     const uint32_t my_bit = 1u << (row / B);  // query block of this row (uniform within a warp)
 #ifdef HEART_TRACE
     const int tr0 = t ? 16 : 0;
-    const bool trw = (warp == 2 || warp == 6) && lane == 0;
+    const bool trw = (warp == 0 || warp == 4) && lane == 0;
 #define HEART_TRS(slot)                   \
   do {                                    \
     if (trw) HEART_TR(h, tr0 + (slot));   \
@@ -401,6 +417,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         tmem_wait_st();
       }
+      // The two warps that share an SM sub-partition (same lane quarter, one per stream) take turns
+      // at the exponentials -- stream 0 step n, stream 1 step n, stream 0 step n+1, ... -- so the
+      // special-function unit serves one of them at full rate while the other waits for scores, loads
+      // them or takes maxima: the streams stay out of phase.
       HEART_TRS(4);
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       const uint64_t c2 = pack_f32x2(c, c), neg_m2 = pack_f32x2(neg_m, neg_m);
@@ -439,6 +459,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->p_full[s]);
       HEART_TRS(7);
+#ifdef HEART_TRACE
+      if (lane == 0) HEART_TR(h, 24 + q);      // arrival time of each warp of the warpgroup
+      if (lane == 0) HEART_TR(h, 28 + q - 0);  // (overwritten below with the s_full time)
+#endif
     }
     // epilogue: the two warpgroups exchange (max, sum) of their streams; warpgroup t then writes
     // output dims [64t, 64t+64) of every row from both accumulators
@@ -495,7 +519,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   // ------------------------------------------------------------------ tear-down
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kWarpQK0) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }

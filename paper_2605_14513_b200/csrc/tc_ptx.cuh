@@ -80,6 +80,22 @@ __device__ __forceinline__ bool elect_one() {
   return pred != 0;
 }
 
+// The same for a waiter with slack (a producer far ahead of its consumer): it sleeps between polls,
+// so that its polling does not compete with the warps that share its scheduler.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t *bar, uint32_t parity, volatile int *abort) {
+  if (mbar_test_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    __nanosleep(256);
+    if (mbar_test_wait(bar, parity)) return true;
+    if (*abort) return false;
+    if (clock64() - t0 > kWaitLimitCycles) {
+      *abort = 1;
+      return false;
+    }
+  }
+}
+
 // ---------------------------------------------------------------- TMA (tiled, 4-D, no multicast)
 __device__ __forceinline__ void tma_load_4d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int c0,
                                             int c1, int c2, int c3) {
