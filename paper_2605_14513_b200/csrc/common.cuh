@@ -34,7 +34,8 @@ __host__ inline void set_chunks(Geom &g) {
 
 // Workspace layout (all offsets 256-byte aligned).
 struct Workspace {
-  int32_t *status;    // [64]   word 0: sticky device-check code; word 1: detail
+  int32_t *status;    // [64]   word 0: sticky device-check code; word 1: detail; word 8: ticket counter
+                      //        of the drift kernel (zero between launches)
   double *bsum;       // [2][R][nb][D]  per-block sums of Q (0) and K (1)
   double *psum;       // [2][R][nchunks][D]  per-CTA partial token sums
   double *mean;       // [2][R][D]      token means of the current step

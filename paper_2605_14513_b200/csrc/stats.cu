@@ -25,7 +25,8 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 
 // One CTA per (chunk of consecutive blocks, head row r, tensor z).  256 threads: 16 row groups x 16
 // chunks of 8 dims.  The 128-bit loads of block i+1 are issued before block i is reduced, so every
-// thread keeps BLOCK/16 loads in flight across the shared-memory combine.
+// thread keeps BLOCK/16 loads in flight across the shared-memory combine; the combine is double-
+// buffered (fp32, the precision the partials have anyway), so a block costs one barrier.
 template <int BLOCK>
 __global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restrict__ Q,
                                                          const uint16_t *__restrict__ K, long long sb,
@@ -37,7 +38,7 @@ __global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restr
   const int c = threadIdx.x & 15, g = threadIdx.x >> 4;
   const uint16_t *X = (z ? K : Q) + (long long)(r / H) * sb + (long long)(r % H) * sh + c * 8;
   const int i0 = chunk * bpc, i1 = min(nb, i0 + bpc);
-  __shared__ double sm[16][kD];
+  __shared__ float sm[2][16][kD];
 
   uint4 cur[ITERS], nxt[ITERS];
   auto load_block = [&](int I, uint4 (&v)[ITERS]) {
@@ -49,9 +50,18 @@ __global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restr
       v[it] = (row < rows) ? ldg_nc_v4(base + (long long)row * sn) : make_uint4(0, 0, 0, 0);
     }
   };
+  // threads 0..127: sum of dim threadIdx.x over the 16 row groups of block I (staged in sm[buf])
+  auto finish_block = [&](int I, int buf, double &total) {
+    double s = 0.0;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) s += (double)sm[buf][k][threadIdx.x];
+    bsum[(((size_t)z * R + r) * nb + I) * kD + threadIdx.x] = s;
+    total += s;
+  };
   load_block(i0, cur);
   double total = 0.0;  // threads 0..127: running token sum of dim threadIdx.x over this CTA's blocks
-  for (int I = i0; I < i1; ++I) {
+  int buf = 0;
+  for (int I = i0; I < i1; ++I, buf ^= 1) {
     if (I + 1 < i1) load_block(I + 1, nxt);
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -65,30 +75,82 @@ __global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restr
       acc[6] += bf16_lo(cur[it].w);
       acc[7] += bf16_hi(cur[it].w);
     }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) sm[g][c * 8 + e] = (double)acc[e];
+    // sm[buf] was last read two blocks ago, before the barrier of the previous block
+    *reinterpret_cast<float4 *>(&sm[buf][g][c * 8]) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    *reinterpret_cast<float4 *>(&sm[buf][g][c * 8 + 4]) = make_float4(acc[4], acc[5], acc[6], acc[7]);
     __syncthreads();
-    if (threadIdx.x < kD) {
-      double s = 0.0;
-#pragma unroll
-      for (int k = 0; k < 16; ++k) s += sm[k][threadIdx.x];
-      bsum[(((size_t)z * R + r) * nb + I) * kD + threadIdx.x] = s;
-      total += s;
-    }
-    __syncthreads();
+    if (threadIdx.x < kD) finish_block(I, buf, total);
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) cur[it] = nxt[it];
   }
   if (threadIdx.x < kD) psum[(((size_t)z * R + r) * gridDim.x + chunk) * kD + threadIdx.x] = total;
 }
 
+// Decision inputs that the last CTA of mean_drift_kernel needs.
+struct DecideArgs {
+  int B, H;
+  const double *delta;
+  double gate_lo, gate_hi;
+  unsigned flags;
+  double *anchor_q, *anchor_k;
+  uint8_t *has_anchor, *refresh_ws;
+  double *drift_out;
+  uint8_t *refresh_out;
+  int *ticket;  // zero between launches
+};
+
+// Head-wise rule, gate over the H heads of batch entry b, anchor update.  One CTA, any block size.
+// `part` and `mean` were written by other CTAs of the same launch: read them past L1.
+__device__ void decide_batch_entry(int b, int R, const double *part, const double *mean, const DecideArgs &a,
+                                   uint8_t *sh_flags /* [2*H] */, int *cnt /* shared */) {
+  const int H = a.H;
+  if (threadIdx.x == 0) *cnt = 0;
+  __syncthreads();
+  for (int h = threadIdx.x; h < H; h += blockDim.x) {
+    const int r = b * H + h;
+    const bool had = a.has_anchor[r] != 0;
+    const double dr = had ? (__ldcg(&part[r]) + __ldcg(&part[R + r])) : __longlong_as_double(0x7ff0000000000000LL);
+    bool rf = !had || (dr > a.delta[r]);
+    if (a.flags & HEART_FORCE_REFRESH) rf = true;
+    sh_flags[h] = rf;
+    sh_flags[H + h] = had;
+    if (a.drift_out) a.drift_out[r] = dr;
+    if (rf) atomicAdd(cnt, 1);
+  }
+  __syncthreads();
+  const double f = (double)*cnt / (double)H;
+  for (int h = threadIdx.x; h < H; h += blockDim.x) {
+    bool rf = sh_flags[h];
+    if (f < a.gate_lo) {
+      if (sh_flags[H + h]) rf = false;
+    } else if (f > a.gate_hi) {
+      rf = true;
+    }
+    sh_flags[h] = rf;
+    const int r = b * H + h;
+    a.refresh_ws[r] = rf;
+    if (a.refresh_out) a.refresh_out[r] = rf;
+    if (rf) a.has_anchor[r] = 1;
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < H * kD; e += blockDim.x) {
+    const int h = e / kD, r = b * H + h;
+    if (sh_flags[h]) {
+      a.anchor_q[(size_t)r * kD + (e % kD)] = __ldcg(&mean[(size_t)r * kD + (e % kD)]);
+      a.anchor_k[(size_t)r * kD + (e % kD)] = __ldcg(&mean[((size_t)R + r) * kD + (e % kD)]);
+    }
+  }
+  __syncthreads();
+}
+
 // One CTA per (head row r, tensor z), 1024 threads = 8 ranges of partial sums x 128 dims.
 // mean[z][r][d] = (sum over the per-CTA partials, ascending) / N;  part[z][r] = sum_d |anchor - mean|.
+// The CTA that finishes last (a ticket counter) then takes the decisions of Algorithm 1 for every
+// batch entry, so drift and decision are one launch.
 __global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restrict__ psum, int R, int N,
-                                                          int nchunks, const double *__restrict__ anchor_q,
-                                                          const double *__restrict__ anchor_k,
-                                                          double *__restrict__ mean,
-                                                          double *__restrict__ part) {
+                                                          int nchunks, double *__restrict__ mean,
+                                                          double *__restrict__ part, const DecideArgs a) {
+  extern __shared__ uint8_t sh_flags[];  // [2*H]: decision, had_anchor
   const int r = blockIdx.x, z = blockIdx.y;
   const int d = threadIdx.x & (kD - 1), grp = threadIdx.x >> 7;  // 8 groups
   const int per = (nchunks + 7) / 8;
@@ -99,6 +161,7 @@ __global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restri
   for (int i = i0; i < i1; ++i) s += src[(size_t)i * kD];
   __shared__ double sm[8][kD];
   __shared__ double red[kD];
+  __shared__ int last, cnt;
   sm[grp][d] = s;
   __syncthreads();
   if (threadIdx.x < kD) {
@@ -107,67 +170,25 @@ __global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restri
     for (int k = 0; k < 8; ++k) t += sm[k][d];
     const double m = t / (double)N;
     mean[((size_t)z * R + r) * kD + d] = m;
-    const double a = (z ? anchor_k : anchor_q)[(size_t)r * kD + d];
-    red[d] = fabs(a - m);
+    const double anc = (z ? a.anchor_k : a.anchor_q)[(size_t)r * kD + d];
+    red[d] = fabs(anc - m);
   }
   __syncthreads();
   for (int w = kD / 2; w > 0; w >>= 1) {  // fixed-shape tree: deterministic
     if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
     __syncthreads();
   }
-  if (threadIdx.x == 0) part[(size_t)z * R + r] = red[0];
-}
-
-// One CTA per batch entry: head-wise rule, gate over the H heads, anchor update.
-__global__ void __launch_bounds__(128) decide_kernel(int H, int R, const double *__restrict__ part,
-                                                     const double *__restrict__ mean,
-                                                     const double *__restrict__ delta, double gate_lo,
-                                                     double gate_hi, unsigned flags,
-                                                     double *__restrict__ anchor_q,
-                                                     double *__restrict__ anchor_k,
-                                                     uint8_t *__restrict__ has_anchor,
-                                                     uint8_t *__restrict__ refresh_ws,
-                                                     double *__restrict__ drift_out,
-                                                     uint8_t *__restrict__ refresh_out) {
-  extern __shared__ uint8_t sh_flags[];  // [2*H]: decision, had_anchor
-  __shared__ int cnt;
-  const int b = blockIdx.x;
-  if (threadIdx.x == 0) cnt = 0;
-  __syncthreads();
-  for (int h = threadIdx.x; h < H; h += blockDim.x) {
-    const int r = b * H + h;
-    const bool had = has_anchor[r] != 0;
-    const double dr = had ? (part[r] + part[R + r]) : __longlong_as_double(0x7ff0000000000000LL);
-    bool rf = !had || (dr > delta[r]);
-    if (flags & HEART_FORCE_REFRESH) rf = true;
-    sh_flags[h] = rf;
-    sh_flags[H + h] = had;
-    if (drift_out) drift_out[r] = dr;
-    if (rf) atomicAdd(&cnt, 1);
+  if (threadIdx.x == 0) {
+    part[(size_t)z * R + r] = red[0];
+    __threadfence();
+    last = (atomicAdd(a.ticket, 1) == (int)(gridDim.x * gridDim.y) - 1);
   }
   __syncthreads();
-  const double f = (double)cnt / (double)H;
-  for (int h = threadIdx.x; h < H; h += blockDim.x) {
-    bool rf = sh_flags[h];
-    if (f < gate_lo) {
-      if (sh_flags[H + h]) rf = false;
-    } else if (f > gate_hi) {
-      rf = true;
-    }
-    sh_flags[h] = rf;
-    const int r = b * H + h;
-    refresh_ws[r] = rf;
-    if (refresh_out) refresh_out[r] = rf;
-    if (rf) has_anchor[r] = 1;
-  }
-  __syncthreads();
-  for (int e = threadIdx.x; e < H * kD; e += blockDim.x) {
-    const int h = e / kD, r = b * H + h;
-    if (sh_flags[h]) {
-      anchor_q[(size_t)r * kD + (e % kD)] = mean[(size_t)r * kD + (e % kD)];
-      anchor_k[(size_t)r * kD + (e % kD)] = mean[((size_t)R + r) * kD + (e % kD)];
-    }
-  }
+  if (!last) return;
+  // Every other CTA has read the old anchors and published its mean and drift part.
+  __threadfence();
+  for (int b = 0; b < a.B; ++b) decide_batch_entry(b, R, part, mean, a, sh_flags, &cnt);
+  if (threadIdx.x == 0) *a.ticket = 0;
 }
 
 cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, const Workspace &w,
@@ -184,14 +205,21 @@ cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, const
 
 cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta, heart_state st,
                           double *drift_out, uint8_t *refresh_out, cudaStream_t s, int *launches) {
-  mean_drift_kernel<<<dim3(g.R, 2), 1024, 0, s>>>(w.psum, g.R, g.N, g.nchunks, st.anchor_q, st.anchor_k,
-                                                  w.mean, w.part);
-  ++*launches;
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  decide_kernel<<<g.B, 128, 2 * g.H, s>>>(g.H, g.R, w.part, w.mean, delta, g.gate_lo, g.gate_hi,
-                                          g.flags, st.anchor_q, st.anchor_k, st.has_anchor, w.refresh,
-                                          drift_out, refresh_out);
+  DecideArgs a;
+  a.B = g.B;
+  a.H = g.H;
+  a.delta = delta;
+  a.gate_lo = g.gate_lo;
+  a.gate_hi = g.gate_hi;
+  a.flags = g.flags;
+  a.anchor_q = st.anchor_q;
+  a.anchor_k = st.anchor_k;
+  a.has_anchor = st.has_anchor;
+  a.refresh_ws = w.refresh;
+  a.drift_out = drift_out;
+  a.refresh_out = refresh_out;
+  a.ticket = w.status + 8;
+  mean_drift_kernel<<<dim3(g.R, 2), 1024, 2 * g.H, s>>>(w.psum, g.R, g.N, g.nchunks, w.mean, w.part, a);
   ++*launches;
   return cudaGetLastError();
 }
