@@ -135,9 +135,15 @@ int heart_step(const heart_config *cfg, const void *Q, const void *K, const void
  *   Q_host, K_host, V_host: bf16, contiguous [B,H,N,D] (cfg strides must be 0,0,0), ideally pinned;
  *   O_host: bf16 [B,H,N,D] result; drift_host [R] fp64 and refresh_host [R] u8 may be NULL.
  *   Q_dev, K_dev, V_dev, O_dev: caller-owned DEVICE staging buffers of B*H*N*D bf16 each.
- * Enqueues on `stream`: three host-to-device copies, the step, the device-to-host copies of O,
- * drift and refresh.  Does not synchronise: the host results are valid once `stream` has drained.
- * delta, tau, st, workspace are device-side exactly as in heart_step. */
+ * Enqueues the uploads of Q and K and the drift / mask kernels on `stream`; V goes up, one group of
+ * heads at a time, on an internal stream while those run, the attention of a head group starts on
+ * `stream` when its V has landed, and its O goes down on a second internal stream while the next
+ * group computes; drift and refresh follow.  `stream` finally waits for the last download.  Does
+ * not synchronise: the host results are valid once `stream` has drained, and later work on `stream`
+ * is ordered after everything this call enqueued.  Results equal heart_step on the same data.
+ * The two internal streams and a few events are created on the first call on each device and kept
+ * (no device memory is allocated); calls on one device are serialised on a host mutex while they
+ * enqueue.  delta, tau, st, workspace are device-side exactly as in heart_step. */
 int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_host, const void *V_host,
                     const double *delta, const double *tau, heart_state *st, void *O_host,
                     double *drift_host, uint8_t *refresh_host, void *Q_dev, void *K_dev, void *V_dev,

@@ -83,6 +83,7 @@ struct AttnParams {
   int32_t *status;
   long long sb, sh, sn;
   int H, N, nb, idx_stride, n_ctas_per_head, dense;
+  int h0, hcount, R_all;  // this launch covers heads [h0, h0 + hcount) of every batch entry; R_all = B*H
   float scale_log2;
 };
 
@@ -123,13 +124,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   volatile int *abort = &bars->abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int r = blockIdx.x / p.n_ctas_per_head, cta_in_head = blockIdx.x % p.n_ctas_per_head;
-  const int bidx = r / p.H, hidx = r % p.H;
+  const int rr = blockIdx.x / p.n_ctas_per_head, cta_in_head = blockIdx.x % p.n_ctas_per_head;
+  const int bidx = rr / p.hcount, hidx = p.h0 + rr % p.hcount;
+  const int r = bidx * p.H + hidx;
   const int row0 = cta_in_head * 128;  // first query token of this CTA
   const int nb = p.nb;
 #ifdef HEART_TRACE
   long long *trace_base = (blockIdx.x == 0 && p.lse != nullptr)
-                              ? reinterpret_cast<long long *>(p.lse + (size_t)(gridDim.x / p.n_ctas_per_head) * p.N)
+                              ? reinterpret_cast<long long *>(p.lse + (size_t)p.R_all * p.N)
                               : nullptr;
 #endif
 
@@ -565,7 +567,7 @@ cudaError_t launch_bk(const Geom &g, const CUtensorMap &mq, const CUtensorMap &m
   const int smem = AttnSmem<B>::TOTAL + 1024;
   cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  attn_tc_kernel<B><<<g.R * prm.n_ctas_per_head, kAttnThreads, smem, s>>>(mq, mk, mv, prm);
+  attn_tc_kernel<B><<<g.B * prm.hcount * prm.n_ctas_per_head, kAttnThreads, smem, s>>>(mq, mk, mv, prm);
   return cudaGetLastError();
 }
 
@@ -573,7 +575,11 @@ cudaError_t launch_bk(const Geom &g, const CUtensorMap &mq, const CUtensorMap &m
 
 cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const void *V,
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,
-                             float *lse, int32_t *status, cudaStream_t s, int *launches) {
+                             float *lse, int32_t *status, cudaStream_t s, int *launches, int h0, int hcount) {
+  if (hcount <= 0) {
+    h0 = 0;
+    hcount = g.H;
+  }
   CUtensorMap mq, mk, mv;
   if (!make_map(&mq, Q, g, 128) || !make_map(&mk, K, g, kStep) || !make_map(&mv, V, g, kStep))
     return cudaErrorInvalidValue;
@@ -592,6 +598,9 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
   prm.idx_stride = g.idx_stride;
   prm.n_ctas_per_head = (g.N + 127) / 128;
   prm.dense = dense ? 1 : 0;
+  prm.h0 = h0;
+  prm.hcount = hcount;
+  prm.R_all = g.R;
   prm.scale_log2 = (float)(g.scale * 1.4426950408889634);
   ++*launches;
   return g.block == 64 ? launch_bk<64>(g, mq, mk, mv, prm, s) : launch_bk<128>(g, mq, mk, mv, prm, s);

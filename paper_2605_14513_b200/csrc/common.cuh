@@ -80,9 +80,11 @@ cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta
                           double *drift_out, uint8_t *refresh_out, cudaStream_t s, int *launches);
 cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
                                 const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches);
+// h0/hcount select the heads [h0, h0 + hcount) of every batch entry (hcount <= 0: all heads).
 cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const void *V,
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,
-                             float *lse, int32_t *status, cudaStream_t s, int *launches);
+                             float *lse, int32_t *status, cudaStream_t s, int *launches, int h0 = 0,
+                             int hcount = 0);
 
 cudaError_t launch_token_drift(const Geom &g, const void *Qa, const void *Ka, const void *Qb,
                                const void *Kb, double *partial, double *drift_out, cudaStream_t s,

@@ -1,6 +1,8 @@
 // C ABI of the HEART hot path: argument validation, workspace carving and kernel sequencing.
 // No device memory is allocated here and nothing synchronises except heart_get_status.
 #include <math.h>
+
+#include <mutex>
 #include <stdio.h>
 #include <string.h>
 
@@ -180,6 +182,46 @@ int heart_step(const heart_config *cfg, const void *Q, const void *K, const void
   return HEART_OK;
 }
 
+namespace {
+
+// Streams and events of heart_step_host, created on first use on each device and kept.
+constexpr int kHostGroups = 4;  // head groups the V copy, the attention and the O copy are pipelined over
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_qk = nullptr, ev_join = nullptr, ev_v[kHostGroups] = {}, ev_o[kHostGroups] = {};
+};
+constexpr int kMaxPipeDevices = 64;
+std::mutex g_pipe_mu;
+HostPipe g_pipe[kMaxPipeDevices];
+
+cudaError_t pipe_for_current_device(HostPipe **out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxPipeDevices) return cudaErrorInvalidDevice;
+  HostPipe &p = g_pipe[dev];
+  if (!p.ready) {
+    if ((e = cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaEventCreateWithFlags(&p.ev_qk, cudaEventDisableTiming)) != cudaSuccess) return e;
+    if ((e = cudaEventCreateWithFlags(&p.ev_join, cudaEventDisableTiming)) != cudaSuccess) return e;
+    for (int i = 0; i < kHostGroups; ++i) {
+      if ((e = cudaEventCreateWithFlags(&p.ev_v[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+      if ((e = cudaEventCreateWithFlags(&p.ev_o[i], cudaEventDisableTiming)) != cudaSuccess) return e;
+    }
+    p.ready = true;
+  }
+  *out = &p;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+// Pipeline: Q and K go up on `stream`, then drift and mask prediction run there while V goes up on
+// an internal stream, one group of heads at a time; the attention of a head group starts when its V
+// has landed and its O goes down on a second internal stream while the next group computes.  `stream`
+// finally waits for the last download, so everything is ordered before later work on `stream`.
 int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_host, const void *V_host,
                     const double *delta, const double *tau, heart_state *st, void *O_host,
                     double *drift_host, uint8_t *refresh_host, void *Q_dev, void *K_dev, void *V_dev,
@@ -196,18 +238,61 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
     return HEART_ERR_INVALID;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   Workspace w = carve(g, workspace);
-  const size_t bytes = sizeof(uint16_t) * (size_t)g.R * g.N * kD;
-  cudaError_t e = cudaMemcpyAsync(Q_dev, Q_host, bytes, cudaMemcpyHostToDevice, s);
+  std::lock_guard<std::mutex> lock(g_pipe_mu);  // the events are shared by the calls on a device
+  HostPipe *pp = nullptr;
+  cudaError_t e = pipe_for_current_device(&pp);
+  if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (streams)");
+  const size_t head_bytes = sizeof(uint16_t) * (size_t)g.N * kD;
+  const size_t bytes = head_bytes * g.R;
+  g_launches = 0;
+  e = cudaMemcpyAsync(Q_dev, Q_host, bytes, cudaMemcpyHostToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(K_dev, K_host, bytes, cudaMemcpyHostToDevice, s);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(V_dev, V_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e == cudaSuccess) e = cudaEventRecord(pp->ev_qk, s);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(pp->s_in, pp->ev_qk, 0);  // V queues behind Q and K
   if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (host to device)");
-  rc = heart_step(cfg, Q_dev, K_dev, V_dev, delta, tau, st, O_dev, nullptr, w.drift, nullptr, workspace, stream);
-  if (rc != HEART_OK) return rc;
-  e = cudaMemcpyAsync(O_host, O_dev, bytes, cudaMemcpyDeviceToHost, s);
-  if (e == cudaSuccess && drift_host)
-    e = cudaMemcpyAsync(drift_host, w.drift, sizeof(double) * (size_t)g.R, cudaMemcpyDeviceToHost, s);
+  const bool dense = (g.flags & HEART_FORCE_DENSE) != 0;
+  if (dense) {
+    fill_dense_outputs_kernel<<<(g.R + 127) / 128, 128, 0, s>>>(g.R, w.drift, nullptr, w.refresh);
+    ++g_launches;
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "fill_dense_outputs");
+  } else {
+    e = launch_block_sums(g, Q_dev, K_dev, w, s, &g_launches);
+    if (e != cudaSuccess) return cuda_fail(e, "block_sums");
+    e = launch_decide(g, w, delta, *st, w.drift, nullptr, s, &g_launches);
+    if (e != cudaSuccess) return cuda_fail(e, "decide");
+    e = launch_predict_mask(g, w, tau, w.refresh, *st, s, &g_launches);
+    if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
+  }
+  const int groups = g.H < kHostGroups ? g.H : kHostGroups;
+  for (int gi = 0; gi < groups; ++gi) {
+    const int h0 = (int)((long long)g.H * gi / groups), h1 = (int)((long long)g.H * (gi + 1) / groups);
+    for (int b = 0; b < g.B && e == cudaSuccess; ++b) {  // one copy per batch entry: its heads h0..h1 are contiguous
+      const size_t off = ((size_t)b * g.H + h0) * head_bytes;
+      e = cudaMemcpyAsync(static_cast<char *>(V_dev) + off, static_cast<const char *>(V_host) + off,
+                          head_bytes * (h1 - h0), cudaMemcpyHostToDevice, pp->s_in);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(pp->ev_v[gi], pp->s_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s, pp->ev_v[gi], 0);
+    if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (host to device)");
+    e = launch_attention(g, Q_dev, K_dev, V_dev, dense ? nullptr : st->kv_idx, dense ? nullptr : st->kv_cnt, dense,
+                         O_dev, nullptr, w.status, s, &g_launches, h0, h1 - h0);
+    if (e != cudaSuccess) return cuda_fail(e, "attention");
+    e = cudaEventRecord(pp->ev_o[gi], s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(pp->s_out, pp->ev_o[gi], 0);
+    for (int b = 0; b < g.B && e == cudaSuccess; ++b) {
+      const size_t off = ((size_t)b * g.H + h0) * head_bytes;
+      e = cudaMemcpyAsync(static_cast<char *>(O_host) + off, static_cast<const char *>(O_dev) + off,
+                          head_bytes * (h1 - h0), cudaMemcpyDeviceToHost, pp->s_out);
+    }
+    if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (device to host)");
+  }
+  // drift and refresh were final before the first attention launch: ev_o[0] on s_out covers them
+  if (drift_host)
+    e = cudaMemcpyAsync(drift_host, w.drift, sizeof(double) * (size_t)g.R, cudaMemcpyDeviceToHost, pp->s_out);
   if (e == cudaSuccess && refresh_host)
-    e = cudaMemcpyAsync(refresh_host, w.refresh, (size_t)g.R, cudaMemcpyDeviceToHost, s);
+    e = cudaMemcpyAsync(refresh_host, w.refresh, (size_t)g.R, cudaMemcpyDeviceToHost, pp->s_out);
+  if (e == cudaSuccess) e = cudaEventRecord(pp->ev_join, pp->s_out);
+  if (e == cudaSuccess) e = cudaStreamWaitEvent(s, pp->ev_join, 0);
   if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (device to host)");
   return HEART_OK;
 }

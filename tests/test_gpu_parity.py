@@ -125,6 +125,38 @@ def test_step_equals_three_calls_and_checkpoint(heart, oracle):
         b.advance()
 
 
+@pytest.mark.parametrize("B,H,flags", [(1, 3, 0), (2, 5, 0), (1, 2, 2)])
+def test_host_buffer_step_equals_device_step(heart, oracle, B, H, flags):
+    """heart_step_host (uploads, per-head-group pipeline, downloads) against heart_step on the same
+    bytes: identical O, drift, refresh and state at every step; the last row of flags runs the dense
+    warm-up mode."""
+    rs = np.random.RandomState(B * 10 + H)
+    wl = inputs.small_workload(H=H, B=B, grid=(3, 10, 14), block=64, seed=33, steps=3,
+                               eps=list(np.exp(rs.uniform(np.log(0.005), np.log(0.3), B * H))),
+                               delta=[0.6] * (B * H))
+    a = Pair(wl, heart, oracle)
+    b = Pair(wl, heart, oracle)
+    staging = tuple(torch.empty_like(b.Q) for _ in range(4))
+    for t in range(3):
+        O, _, drift, refresh = a.gpu_step(flags=flags, want_lse=False)
+        b.cfg.flags = flags
+        host = [x.cpu().contiguous().pin_memory() for x in (b.Q, b.K, b.V)]
+        Oh = torch.full(b.Q.shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+        dh = torch.full((wl.R,), float("nan"), dtype=torch.float64).pin_memory()
+        rh = torch.full((wl.R,), 7, dtype=torch.uint8).pin_memory()
+        heart.heart_step_host(b.cfg, host[0], host[1], host[2], b.delta, b.tau, b.gst, Oh, staging, b.ws,
+                              drift_host=dh, refresh_host=rh)
+        torch.cuda.current_stream().synchronize()  # the call's own ordering: no device-wide sync
+        assert heart.heart_get_status(b.ws) == 0
+        assert np.array_equal(drift, dh.numpy()) and np.array_equal(refresh, rh.numpy())
+        Oc = O.cpu()
+        assert torch.equal(Oc.view(torch.int16), Oh.view(torch.int16))
+        for x, y in zip(a.gst.tensors(), b.gst.tensors()):
+            assert torch.equal(x, y)
+        a.advance()
+        b.advance()
+
+
 def test_run_to_run_bit_reproducible(heart, oracle):
     wl = inputs.small_workload(H=2, grid=(3, 10, 14), block=64, seed=5)
     outs = []
