@@ -8,8 +8,9 @@
 // tile of scores.  Phase 2 gives each
 // warp two rows: two-pass softmax, then top-p WITHOUT a sort: the kept set is {p > theta} plus the
 // lowest-index ties at theta, where theta is the largest element value whose ">= theta" mass still
-// reaches tau -- found by a 62-step bit-wise search over the IEEE-754 pattern of p (positive
-// doubles order like their bit patterns).  Everything is fp64 so the integer outputs (bit mask,
+// reaches tau -- found by a search over the IEEE-754 pattern of p (positive doubles order like
+// their bit patterns): the top 14 bits two at a time over all blocks, the rest directly over the
+// few blocks that share that prefix.  Everything is fp64 so the integer outputs (bit mask,
 // ascending index list, count) agree with a plain fp64 sort-and-accumulate reference except when
 // the cumulative mass is within rounding (1e-15) of tau.
 #include <type_traits>
@@ -184,10 +185,37 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
         }
         return warp_sum((g0 + g1) + (g2 + g3));
       };
-      constexpr int kSplit = 48;  // bits [kSplit, 62) are searched over all blocks
-      for (int bit = 61; bit >= kSplit; --bit) {
-        const long long cand = theta | (1LL << bit);
-        if (mass_at_least(cand) >= t) theta = cand;
+      constexpr int kSplit = 48;  // bits [kSplit, 62) are searched over all blocks, two bits a round
+      // (three trial thresholds per round: their three reductions run side by side)
+      auto masses_at_least = [&](long long c1, long long c2, long long c3, double &m1, double &m2, double &m3) {
+        double a1 = 0.0, a2 = 0.0, a3 = 0.0, b1 = 0.0, b2 = 0.0, b3 = 0.0;  // fixed split: same order on every run
+#pragma unroll
+        for (int j = 0; j < NJ; j += 2) {
+          const long long k0 = __double_as_longlong(p[j]), k1 = __double_as_longlong(p[j + 1]);
+          if (k0 >= c1) a1 += p[j];
+          if (k0 >= c2) a2 += p[j];
+          if (k0 >= c3) a3 += p[j];
+          if (k1 >= c1) b1 += p[j + 1];
+          if (k1 >= c2) b2 += p[j + 1];
+          if (k1 >= c3) b3 += p[j + 1];
+        }
+        m1 = a1 + b1;
+        m2 = a2 + b2;
+        m3 = a3 + b3;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          m1 += __shfl_xor_sync(0xffffffffu, m1, o);
+          m2 += __shfl_xor_sync(0xffffffffu, m2, o);
+          m3 += __shfl_xor_sync(0xffffffffu, m3, o);
+        }
+      };
+      static_assert((62 - kSplit) % 2 == 0 && NJ % 2 == 0, "two bits per round, two blocks per step");
+      for (int bit = 60; bit >= kSplit; bit -= 2) {
+        // trial patterns theta | 01, 10, 11 at bits (bit+1, bit): the mass is non-increasing in them
+        const long long c1 = theta | (1LL << bit), c2 = theta | (2LL << bit), c3 = theta | (3LL << bit);
+        double m1, m2, m3;
+        masses_at_least(c1, c2, c3, m1, m2, m3);
+        theta = (m3 >= t) ? c3 : (m2 >= t) ? c2 : (m1 >= t) ? c1 : theta;
       }
       // ... then only the blocks whose pattern shares that prefix can still decide the remaining bits:
       // they are compacted (through this row's no longer needed score slots) and the other 48 rounds
@@ -211,13 +239,29 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
       const double mass_above = warp_sum(ab0 + ab1);
       __syncwarp();
       if (n_cand <= 64) {
+        // Few candidates: each lane takes two of them and adds up, over all candidates, the mass at
+        // or above its own value; theta is the largest candidate whose mass still reaches tau (the
+        // smallest candidate always does: that is what the prefix search established).
         const double c0 = (lane < n_cand) ? scr[lane] : 0.0, c1 = (lane + 32 < n_cand) ? scr[lane + 32] : 0.0;
         const long long k0 = __double_as_longlong(c0), k1 = __double_as_longlong(c1);
-        for (int bit = kSplit - 1; bit >= 0; --bit) {
-          const long long cand = theta | (1LL << bit);
-          const double g = mass_above + warp_sum((k0 >= cand ? c0 : 0.0) + (k1 >= cand ? c1 : 0.0));
-          if (g >= t) theta = cand;
+        double g0 = mass_above, g1 = mass_above;
+        long long k_min = 0x7fffffffffffffffLL;
+        for (int n = 0; n < n_cand; ++n) {
+          const double v = scr[n];
+          const long long kv = __double_as_longlong(v);
+          if (kv >= k0) g0 += v;
+          if (kv >= k1) g1 += v;
+          k_min = kv < k_min ? kv : k_min;
         }
+        long long best = k_min;
+        if (lane < n_cand && g0 >= t && k0 > best) best = k0;
+        if (lane + 32 < n_cand && g1 >= t && k1 > best) best = k1;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const long long other = __shfl_xor_sync(0xffffffffu, best, o);
+          best = other > best ? other : best;
+        }
+        theta = best;
       } else {  // many near-equal blocks: keep searching over all of them
         for (int bit = kSplit - 1; bit >= 0; --bit) {
           const long long cand = theta | (1LL << bit);
