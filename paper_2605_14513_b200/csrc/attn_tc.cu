@@ -71,6 +71,7 @@ struct AttnBars {
   uint64_t pv_done[kStages];                  // P_h V_h complete: V stage and S/P buffer are free
   uint64_t p_full[kStages];                   // P_h written (one arrival per warp of the stream)
   uint32_t tmem_base;
+  int chunk_cnt[32];  // flagged key blocks per 32-block chunk (set-up)
   int n_union;
   int abort;
   int bad;
@@ -136,6 +137,23 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
 #endif
 
   // ------------------------------------------------------------------ set-up
+  if (tid == 0) HEART_TR(62, 0);
+  // The lists of this tile's query blocks come from global memory: their loads are issued first
+  // (speculatively, inside the row pitch) so that their latency overlaps the rest of the set-up.
+  constexpr int kPre = kMaxNb / kAttnThreads;  // entries per thread held in registers
+  int cnt_q[L::QBT];
+  int32_t ent[L::QBT][kPre];
+#pragma unroll
+  for (int qb = 0; qb < L::QBT; ++qb) {
+    const int I = cta_in_head * L::QBT + qb;
+    const size_t row = (size_t)r * nb + I;
+    cnt_q[qb] = (I < nb) ? (p.dense ? nb : p.kv_cnt[row]) : 0;
+#pragma unroll
+    for (int k = 0; k < kPre; ++k) {
+      const int t = tid + k * kAttnThreads;
+      ent[qb][k] = (I < nb && !p.dense && t < p.idx_stride) ? p.kv_idx[row * p.idx_stride + t] : t;
+    }
+  }
   if (tid == 0) {
     mbar_init(&bars->q_full, 1);
     for (int i = 0; i < kStages; ++i) {
@@ -152,22 +170,42 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   }
   for (int j = tid; j < nb; j += kAttnThreads) tbl[j] = 0u;
   __syncthreads();
+  if (warp == kWarpKProd && lane == 0) {  // the Q tile does not depend on the lists: start it now
+    tma_prefetch_desc(&map_q);
+    tma_prefetch_desc(&map_kv);
+    tma_prefetch_desc(&map_v);
+    mbar_expect_tx(&bars->q_full, L::Q_BYTES);
+    tma_load_4d(Qs, &map_q, &bars->q_full, 0, row0, hidx, bidx);
+    tma_load_4d(Qs + 128 * 128, &map_q, &bars->q_full, 64, row0, hidx, bidx);
+  }
+#pragma unroll
   for (int qb = 0; qb < L::QBT; ++qb) {  // scatter: flag bit qb of every key block listed by query block qb
     const int I = cta_in_head * L::QBT + qb;
-    if (I >= nb) break;
-    const size_t row = (size_t)r * nb + I;
-    int cnt = p.dense ? nb : p.kv_cnt[row];
+    int cnt = cnt_q[qb];
     if (cnt < 0 || cnt > p.idx_stride) {
       bars->bad = 1;
       cnt = cnt < 0 ? 0 : p.idx_stride;
     }
-    const int32_t *list = p.kv_idx + row * p.idx_stride;
-    for (int t = tid; t < cnt; t += kAttnThreads) {
-      const int J = p.dense ? t : list[t];
-      if (J < 0 || J >= nb)
-        bars->bad = 1;  // skipped, reported
-      else
-        atomicOr(&tbl[J], 1u << qb);
+#pragma unroll
+    for (int k = 0; k < kPre; ++k) {
+      const int t = tid + k * kAttnThreads;
+      if (t < cnt) {
+        const int J = ent[qb][k];
+        if (J < 0 || J >= nb)
+          bars->bad = 1;  // skipped, reported
+        else
+          atomicOr(&tbl[J], 1u << qb);
+      }
+    }
+    if (cnt > kPre * kAttnThreads) {  // longer than any list of distinct blocks: the slow way
+      const int32_t *list = p.kv_idx + ((size_t)r * nb + I) * p.idx_stride;
+      for (int t = kPre * kAttnThreads + tid; t < cnt; t += kAttnThreads) {
+        const int J = list[t];
+        if (J < 0 || J >= nb)
+          bars->bad = 1;
+        else
+          atomicOr(&tbl[J], 1u << qb);
+      }
     }
   }
   if (warp == kWarpQK0) {
@@ -175,26 +213,42 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     tmem_relinquish();
   }
   __syncthreads();
-  if (warp == kWarpKProd) {  // ascending compaction of the flagged key blocks
-    int count = 0;
-    for (int base = 0; base < nb; base += 32) {
-      const int J = base + lane;
-      const uint32_t f = (J < nb) ? tbl[J] : 0u;
-      const unsigned ballot = __ballot_sync(0xffffffffu, f != 0u);
-      if (f != 0u) uni[count + __popc(ballot & ((1u << lane) - 1u))] = J | (int)(f << 16);
-      count += __popc(ballot);
+  {  // ascending compaction of the flagged key blocks: warp w takes the 32-block chunks w, w+16
+    constexpr int kChunksPerWarp = kMaxNb / 32 / (kAttnThreads / 32);
+    uint32_t f[kChunksPerWarp];
+    unsigned ballot[kChunksPerWarp];
+#pragma unroll
+    for (int i = 0; i < kChunksPerWarp; ++i) {
+      const int J = (warp + i * (kAttnThreads / 32)) * 32 + lane;
+      f[i] = (J < nb) ? tbl[J] : 0u;
+      ballot[i] = __ballot_sync(0xffffffffu, f[i] != 0u);
+      if (lane == 0) bars->chunk_cnt[warp + i * (kAttnThreads / 32)] = __popc(ballot[i]);
     }
-    if (lane == 0) {
-      bars->n_union = count;
+    __syncthreads();
+    // exclusive prefix over the 32 chunk counts (every warp computes it: lane = chunk)
+    const int mine = bars->chunk_cnt[lane];
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+#pragma unroll
+    for (int i = 0; i < kChunksPerWarp; ++i) {
+      const int chunk = warp + i * (kAttnThreads / 32);
+      const int base = __shfl_sync(0xffffffffu, incl - mine, chunk);
+      if (f[i] != 0u) uni[base + __popc(ballot[i] & ((1u << lane) - 1u))] = (chunk * 32 + lane) | (int)(f[i] << 16);
+    }
+    const int total = __shfl_sync(0xffffffffu, incl, 31);
+    if (tid == 0) {
+      bars->n_union = total;
       if (bars->bad) atomicExch(p.status, HEART_ERR_DEVICE_CHECK);
-      tma_prefetch_desc(&map_q);
-      tma_prefetch_desc(&map_kv);
-      tma_prefetch_desc(&map_v);
     }
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  if (tid == 0) HEART_TR(62, 1);
   const uint32_t tmem = bars->tmem_base;
   const int U = bars->n_union;
   const int NH = U * HPB;  // key steps; step h belongs to stream h & 1
@@ -211,10 +265,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   };
   if (warp >= 8) setmaxnreg_dec<kRegsHelper>();
   if (warp == kWarpKProd) {
-    if (lane == 0) {  // ===== TMA producer: Q once, then K_h into stage h & 3
-      mbar_expect_tx(&bars->q_full, L::Q_BYTES);
-      tma_load_4d(Qs, &map_q, &bars->q_full, 0, row0, hidx, bidx);
-      tma_load_4d(Qs + 128 * 128, &map_q, &bars->q_full, 64, row0, hidx, bidx);
+    if (lane == 0) {  // ===== TMA producer (Q was started during set-up): K_h into stage h & 3
       int issued = 0;
       for (int h = 0; h < NH; ++h) {
         const int s = h & 3, ph = (h >> 2) & 1;
@@ -519,8 +570,10 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   }
 
   // ------------------------------------------------------------------ tear-down
+  if (tid == 0) HEART_TR(62, 2);
   tc_fence_before();
   __syncthreads();
+  if (tid == 0) HEART_TR(62, 3);
   if (warp == kWarpQK0) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
