@@ -269,7 +269,7 @@ def run_ours(args, rank, world):
     if rank == 0:
         peak_tf = pk["bf16_tflops_sustained"]
         # DRAM bytes per attention launch from the ncu capture summarised in profiles/ (this workload only)
-        traffic = {"wan1.3b-480p": 388.1e6}.get(wl.name)
+        traffic = {"wan1.3b-480p": 399.1e6}.get(wl.name)
         roofline = {"kernel": "block-sparse attention", "bound": "tensor", "achieved": attn_tflops, "peak": peak_tf,
                     "unit": "TFLOP/s", "frac": attn_tflops / peak_tf, "traffic": traffic,
                     "peak_source": pk["source"] + " (sustained bf16 cuBLAS, kernel timed inside a long step)",
