@@ -470,10 +470,6 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
         tmem_wait_st();
       }
-      // The two warps that share an SM sub-partition (same lane quarter, one per stream) take turns
-      // at the exponentials -- stream 0 step n, stream 1 step n, stream 0 step n+1, ... -- so the
-      // special-function unit serves one of them at full rate while the other waits for scores, loads
-      // them or takes maxima: the streams stay out of phase.
       HEART_TRS(4);
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       const uint64_t c2 = pack_f32x2(c, c), neg_m2 = pack_f32x2(neg_m, neg_m);
@@ -513,8 +509,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       if (lane == 0) mbar_arrive(&bars->p_full[s]);
       HEART_TRS(7);
 #ifdef HEART_TRACE
-      if (lane == 0) HEART_TR(h, 24 + q);      // arrival time of each warp of the warpgroup
-      if (lane == 0) HEART_TR(h, 28 + q - 0);  // (overwritten below with the s_full time)
+      if (lane == 0) HEART_TR(h, 24 + q);  // arrival time of each warp of the warpgroup
 #endif
     }
     // epilogue: the two warpgroups exchange (max, sum) of their streams; warpgroup t then writes
