@@ -238,6 +238,21 @@ def run_ours(args, rank, world):
     attn_tflops = flops_step / (ms_attn * 1e-3) / 1e12
     stats_bytes = 4.0 * wl.R * wl.N * wl.D  # Q and K read once (bf16)
 
+    # ---- the same attention kernel with a full mask, measured where it fits in time (a dense run of the
+    # two 720P shapes would take 0.1-0.15 s per launch): the sparse path's speedup over its own dense mode
+    dense_ms = None
+    if dense_flops < 3e13:
+        cfg_dense = heart.make_config(wl.B, wl.H, wl.N, wl.block, flags=heart.FORCE_DENSE)
+        Q, Kt, V = steps_in[W]
+        heart.heart_block_sparse_attn(cfg_dense, Q, Kt, V, None, None, O, ws)
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(3):
+            heart.heart_block_sparse_attn(cfg_dense, Q, Kt, V, None, None, O, ws)
+        b_.record()
+        torch.cuda.synchronize()
+        dense_ms = a.elapsed_time(b_) / 3
+
     # ---- end-to-end pass: host (pinned) Q/K/V in, O/drift/refresh out, through heart_step_host
     e2e = None
     if not args.no_e2e:
@@ -289,6 +304,9 @@ def run_ours(args, rank, world):
             "retained_tflops": attn_tflops, "retained_tflops_vs_bf16_peak": attn_tflops / pk["bf16_tflops"],
             "dense_equivalent_tflops": dense_flops / (ms_attn * 1e-3) / 1e12,
             "dense_equivalent_speedup_at_same_throughput": dense_flops / flops_step,
+            "dense_attention_ms_measured": dense_ms,
+            "dense_tflops_measured": (dense_flops / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
+            "attention_speedup_vs_measured_dense": (dense_ms / ms_attn) if dense_ms else None,
             "roofline": roofline,
             "roofline_stats": {"kernel": "block sums + drift (heart_drift)", "bound": "hbm", "achieved": hbm,
                                "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm / pk["hbm_gbs"],
