@@ -5,28 +5,28 @@
 // the half that does not list a key block see -inf there).  Keys are processed 64 at a time: a "key
 // step" is one 64-token block, or one half of a 128-token block.
 //
-// The key steps are dealt to two independent streams (even / odd step index).  Each stream keeps
-// its own running max, row sum and output accumulator (merged at the end) and is served by its own
-// softmax warpgroup, one thread per query row, so the two warpgroups run out of phase: while one
-// computes exponentials the other waits, loads scores or takes maxima, and the special-function
-// unit -- the scarcest resource of this kernel -- stays busy.  Each stream double-buffers its scores
-// in tensor memory: S of the stream's next step is computed while the softmax works on the current
-// one, so the serial chain softmax -> P V -> Q K^T -> softmax is off the critical path.
+// Two CTAs share an SM (256 threads, 105 KB of shared memory and 256 of the 512 tensor-memory
+// columns each).  They work on different query tiles and drift out of phase, so while the softmax
+// warps of one compute exponentials -- the special-function unit is the scarcest resource of this
+// kernel -- those of the other wait, load scores or take maxima, and the set-up and the epilogue of
+// one tile hide behind the key steps of the other.  Inside a CTA the scores are double-buffered in
+// tensor memory: S of step h+1 is complete before the softmax of step h ends, so the serial chain
+// softmax -> P V -> Q K^T -> softmax is off the critical path.
 //
-// Warp roles (512 threads; registers are moved from the helper warps to the softmax warps at start):
-//   warps 0-3   softmax warpgroup of stream 0; warps 4-7 of stream 1.  Per key step a thread reads
+// Warp roles (registers are moved from the helper warps to the softmax warps at start):
+//   warps 0-3   softmax, one thread per query row (lane quarter = warp).  Per key step a thread reads
 //               its row of S (64 columns), takes the max, rescales its row of O only when the max
 //               grew by more than 2^8, writes P = 2^(s*scale*log2e - m) as bf16 over the first half
-//               of the S buffer and adds the row sum.  At the end the two warpgroups exchange
-//               (max, sum), and warpgroup t writes output dims [64t, 64t+64) of every row (and lse).
-//   warp 8      TMA producer for Q (once) and K, through a four-stage shared-memory ring
-//               (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers).
-//   warp 9      TMA producer for V (its own ring: V_h is needed four key steps later than K_h).
-//   warp 10     MMA issuer (one elected lane) of O_t += P_h V_h, P_h read from tensor memory.
-//   warps 12-15 MMA issuers of S_h = Q K_h^T (tcgen05.mma, operands in shared memory), warp 12+i
-//               for the key steps h = i (mod 4).
-// Tensor memory (512 columns): O_0 | O_1 | S[4]  =  128 + 128 + 4 x 64; key step h uses S[h & 3]
-// (stream h & 1, buffer (h >> 1) & 1) and shared-memory stage h & 3; P_h aliases S[h & 3].
+//               of the S buffer and adds the row sum; at the end it writes O / l (and lse).
+//   warps 4-7   one helper role each, rotated with the CTA index so that the two CTAs of an SM
+//               rarely put the same role on the same sub-partition:
+//               K producer  TMA loads of Q (once) and of the listed K blocks into a two-stage ring
+//                           (cp.async.bulk.tensor, 128-byte swizzle, completion on mbarriers);
+//               V producer  the same for V (its own ring: V_h is needed two key steps after K_h);
+//               QK issuer   S_h = Q K_h^T (tcgen05.mma, operands in shared memory), one elected lane;
+//               PV issuer   O += P_h V_h with P_h read from tensor memory.
+// Tensor memory (256 columns per CTA): O | S[2]  =  128 + 2 x 64; key step h uses S[h & 1] and
+// shared-memory stage h & 1; P_h aliases S[h & 1].
 //
 // Every wait is bounded; a wait that runs out raises a CTA-wide abort flag and the status word, the
 // roles drain, tensor memory is freed and the CTA exits.
@@ -38,13 +38,13 @@
 namespace heart {
 using namespace tc;
 
-constexpr int kAttnThreads = 512;
-// warp roles: 0-3 softmax of stream 0, 4-7 softmax of stream 1 (lane quarter = warp & 3), then the
-// helpers, two per SM sub-partition (warp & 3)
-constexpr int kWarpKProd = 8, kWarpVProd = 9, kWarpPV = 10, kWarpQK0 = 12;  // QK issuers: 12..15
-constexpr int kRegsSoftmax = 176, kRegsHelper = 80;  // 2 * (176 + 80) * 32 lanes = one sub-partition
+constexpr int kAttnThreads = 256;
+// warp roles: 0-3 softmax (lane quarter = warp), then one helper per SM sub-partition
+constexpr int kRoleKProd = 0, kRoleVProd = 1, kRolePV = 2, kRoleQK = 3;  // helper warp 4 + ((role + CTA index) & 3)
+constexpr int kRegsSoftmax = 176, kRegsHelper = 80;  // (176 + 80) * 128 threads = the CTA's 256 x 128
 constexpr int kStep = 64;   // keys per key step
-constexpr int kStages = 4;  // K / V ring depth = number of S buffers
+constexpr int kStages = 2;  // K / V ring depth = number of S buffers
+constexpr int kTmemCols = 256;  // O (128) + S[2] (2 x 64): two CTAs share the 512 columns of an SM
 constexpr int kMaxNb = HEART_MAX_BLOCKS;
 
 // Shared-memory plan.
@@ -59,8 +59,7 @@ struct AttnSmem {
   static constexpr int OFF_V = OFF_K + kStages * KV_BYTES;
   static constexpr int OFF_UNI = OFF_V + kStages * KV_BYTES;  // int32[kMaxNb]: J | flags << 16
   static constexpr int OFF_TBL = OFF_UNI + 4 * kMaxNb;        // uint32[kMaxNb]: flags per key block
-  static constexpr int OFF_XCH = OFF_TBL + 4 * kMaxNb;        // float[2 streams][2][128 rows]: max, sum
-  static constexpr int OFF_BAR = OFF_XCH + 2048;              // mbarriers and scalars
+  static constexpr int OFF_BAR = OFF_TBL + 4 * kMaxNb;        // mbarriers and scalars
   static constexpr int TOTAL = OFF_BAR + 512;
 };
 
@@ -109,7 +108,7 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 }
 
 template <int B>
-__global__ void __launch_bounds__(kAttnThreads, 1)
+__global__ void __launch_bounds__(kAttnThreads, 2)
     attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_kv,
                    const __grid_constant__ CUtensorMap map_v, const AttnParams p) {
   using L = AttnSmem<B>;
@@ -120,11 +119,14 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   unsigned char *Qs = smem + L::OFF_Q, *Ks = smem + L::OFF_K, *Vs = smem + L::OFF_V;
   int32_t *uni = reinterpret_cast<int32_t *>(smem + L::OFF_UNI);
   uint32_t *tbl = reinterpret_cast<uint32_t *>(smem + L::OFF_TBL);
-  float *xch = reinterpret_cast<float *>(smem + L::OFF_XCH);
   AttnBars *bars = reinterpret_cast<AttnBars *>(smem + L::OFF_BAR);
   volatile int *abort = &bars->abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // The helper roles rotate with the CTA index: the two CTAs that share an SM then rarely have the
+  // same role (above all the issuer of the score products) on the same sub-partition.
+  const int kWarpKProd = 4 + ((kRoleKProd + blockIdx.x) & 3), kWarpVProd = 4 + ((kRoleVProd + blockIdx.x) & 3),
+            kWarpPV = 4 + ((kRolePV + blockIdx.x) & 3), kWarpQK = 4 + ((kRoleQK + blockIdx.x) & 3);
   const int rr = blockIdx.x / p.n_ctas_per_head, cta_in_head = blockIdx.x % p.n_ctas_per_head;
   const int bidx = rr / p.hcount, hidx = p.h0 + rr % p.hcount;
   const int r = bidx * p.H + hidx;
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       mbar_init(&bars->v_full[i], 1);
       mbar_init(&bars->qk_done[i], 1);
       mbar_init(&bars->pv_done[i], 1);
-      mbar_init(&bars->p_full[i], 4);  // one arrival per warp of the stream's warpgroup
+      mbar_init(&bars->p_full[i], 4);  // one arrival per softmax warp
     }
     bars->abort = 0;
     bars->bad = 0;
@@ -208,8 +210,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       }
     }
   }
-  if (warp == kWarpQK0) {
-    tmem_alloc(&bars->tmem_base, 512);
+  if (warp == kWarpQK) {
+    tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
   }
   __syncthreads();
@@ -251,7 +253,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   if (tid == 0) HEART_TR(62, 1);
   const uint32_t tmem = bars->tmem_base;
   const int U = bars->n_union;
-  const int NH = U * HPB;  // key steps; step h belongs to stream h & 1
+  const int NH = U * HPB;  // key steps; step h uses S buffer and shared-memory stage h & 1
   // first key token of step h
   auto key0_of = [&](int h) -> int { return (uni[h / HPB] & 0xffff) * B + (h % HPB) * kStep; };
 
@@ -263,12 +265,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
     while (!mbar_try_wait(bar, parity) && clock64() - t0 < 40000000LL) {
     }
   };
-  if (warp >= 8) setmaxnreg_dec<kRegsHelper>();
+  if (warp >= 4) setmaxnreg_dec<kRegsHelper>();
   if (warp == kWarpKProd) {
-    if (lane == 0) {  // ===== TMA producer (Q was started during set-up): K_h into stage h & 3
+    if (lane == 0) {  // ===== TMA producer (Q was started during set-up): K_h into stage h & 1
       int issued = 0;
       for (int h = 0; h < NH; ++h) {
-        const int s = h & 3, ph = (h >> 2) & 1;
+        const int s = h % kStages, ph = (h / kStages) & 1;
         // the stage is free once S_{h-4} = Q K_{h-4}^T is complete
         if (h >= kStages && !mbar_wait_relaxed(&bars->qk_done[s], ph ^ 1, abort)) break;
         const int key0 = key0_of(h);
@@ -280,13 +282,13 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       }
       settle(&bars->q_full, 0);  // nobody else waits for Q when the union is empty
       if (*abort)
-        for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->k_full[h & 3], (h >> 2) & 1);
+        for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->k_full[h % kStages], (h / kStages) & 1);
     }
   } else if (warp == kWarpVProd) {
-    if (lane == 0) {  // ===== TMA producer: V_h into stage h & 3
+    if (lane == 0) {  // ===== TMA producer: V_h into stage h & 1
       int issued = 0;
       for (int h = 0; h < NH; ++h) {
-        const int s = h & 3, ph = (h >> 2) & 1;
+        const int s = h % kStages, ph = (h / kStages) & 1;
         if (h >= kStages && !mbar_wait_relaxed(&bars->pv_done[s], ph ^ 1, abort)) break;
         const int key0 = key0_of(h);
         unsigned char *dst = Vs + s * L::KV_BYTES;
@@ -296,14 +298,12 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         issued = h + 1;
       }
       if (*abort)
-        for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->v_full[h & 3], (h >> 2) & 1);
+        for (int h = (issued > kStages ? issued - kStages : 0); h < issued; ++h) settle(&bars->v_full[h % kStages], (h / kStages) & 1);
     }
-  } else if (warp == kWarpPV || warp >= kWarpQK0) {
-    // ===== MMA issuers.  Warp 12+i issues S_h = Q K_h^T for the key steps h = i, i+4, ... (buffer
-    // and stage i); warp 10 issues every O_t += P_h V_h.  An MMA that waits for the tensor pipe
-    // holds up the other warps of its SM sub-partition, so the S products -- eight MMAs per key
-    // step -- rotate over the four sub-partitions.  The whole warp runs the loop (uniform control
-    // flow keeps the descriptors in uniform registers), one elected lane issues.
+  } else if (warp == kWarpPV || warp == kWarpQK) {
+    // ===== MMA issuers: warp 7 issues S_h = Q K_h^T, warp 6 issues O += P_h V_h.  Two warps, so that
+    // the barrier round trips of one overlap the issue of the other.  The whole warp runs the loop
+    // (uniform control flow keeps the descriptors in uniform registers), one elected lane issues.
     if (NH > 0) {
       constexpr uint32_t idesc_qk = idesc_bf16_f32(128, kStep, false, false);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(128, 128, false, true);
@@ -317,56 +317,56 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       };
       const bool leader = elect_one();  // the same lane every time: commits track its MMAs
       bool ok = true;
-      if (warp >= kWarpQK0) {
-        const int s = warp - kWarpQK0;  // S buffer and K stage of this warp
+      if (warp == kWarpQK) {
         const uint64_t q_desc = smem_desc_sw128(smem_u32(Qs), 16, 1024);
-        const uint64_t k_desc = smem_desc_sw128(smem_u32(Ks) + s * L::KV_BYTES, 16, 1024);
-        const uint32_t d = tmem + 256 + s * kStep;
-        auto issue_qk = [&]() {  // S[s] = Q K^T with the K tile that sits in stage s
+        const uint64_t k_desc = smem_desc_sw128(smem_u32(Ks), 16, 1024);
+        auto issue_qk = [&](int s) {  // S[s] = Q K^T with the K tile that sits in stage s
+          const uint32_t d = tmem + 128 + s * kStep;
+          const uint64_t ks_desc = at(k_desc, s * (L::KV_BYTES >> 4));
           if (leader) {
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
-              mma_ss(d, at(q_desc, (ks >> 2) * 1024 + (ks & 3) * 2), at(k_desc, (ks >> 2) * 512 + (ks & 3) * 2), idesc_qk,
-                     ks > 0 ? 1u : 0u);
+              mma_ss(d, at(q_desc, (ks >> 2) * 1024 + (ks & 3) * 2), at(ks_desc, (ks >> 2) * 512 + (ks & 3) * 2),
+                     idesc_qk, ks > 0 ? 1u : 0u);
             tc_commit(&bars->qk_done[s]);
           }
           __syncwarp();
         };
-        if (s < NH) {
-          ok = mbar_wait(&bars->q_full, 0, abort);
-          if (ok) ok = mbar_wait(&bars->k_full[s], 0, abort);
+        ok = mbar_wait(&bars->q_full, 0, abort);
+        for (int h = 0; h < kStages && h < NH && ok; ++h) {
+          ok = mbar_wait(&bars->k_full[h], 0, abort);
           if (ok) {
             tc_fence_after();
-            issue_qk();
+            issue_qk(h);
           }
         }
-        for (int h = s; h + kStages < NH && ok; h += kStages) {
-          const int ph = (h >> 2) & 1;
+        for (int h = 0; h + kStages < NH && ok; ++h) {
+          const int s = h % kStages, ph = (h / kStages) & 1;
           // S[s] holds P_h until the product P_h V_h has read it
           ok = mbar_wait(&bars->k_full[s], ph ^ 1, abort);
           if (ok) ok = mbar_wait(&bars->pv_done[s], ph, abort);
           if (!ok) break;
           HEART_TR(h, 10);
           tc_fence_after();
-          issue_qk();
+          issue_qk(s);
           HEART_TR(h, 11);
         }
       } else {
         const uint64_t v_desc = smem_desc_sw128(smem_u32(Vs), kStep * 128, 1024);
-        for (int h = 0; h < NH && ok; ++h) {  // O_t (+)= P_h V_h, t = h & 1; P_h sits over S[h & 3]
-          const int s = h & 3, ph = (h >> 2) & 1;
+        for (int h = 0; h < NH && ok; ++h) {  // O (+)= P_h V_h; P_h sits over S[h & 1]
+          const int s = h % kStages, ph = (h / kStages) & 1;
           ok = mbar_wait(&bars->v_full[s], ph, abort);
           HEART_TR(h, 12);
           if (ok) ok = mbar_wait(&bars->p_full[s], ph, abort);
           if (!ok) break;
           HEART_TR(h, 8);
           tc_fence_after();
-          const uint32_t d = tmem + (h & 1) * 128, pa = tmem + 256 + s * kStep;
+          const uint32_t d = tmem, pa = tmem + 128 + s * kStep;
           const uint64_t vs_desc = at(v_desc, s * (L::KV_BYTES >> 4));
           if (leader) {
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
-              mma_ts(d, pa + ks * 8, at(vs_desc, ks * 128), idesc_pv, (h >= 2 || ks > 0) ? 1u : 0u);
+              mma_ts(d, pa + ks * 8, at(vs_desc, ks * 128), idesc_pv, (h > 0 || ks > 0) ? 1u : 0u);
             tc_commit(&bars->pv_done[s]);
           }
           __syncwarp();
@@ -374,25 +374,20 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         }
       }
     }
-  } else if (warp >= 8) {
-    // warp 11: no role (it completes the helper warpgroups)
   } else {
-    // ===== softmax / correction / epilogue: warpgroup t owns stream t, thread = one query row
-    // The stream index t is a run-time value (uniform per warp): both warpgroups run one copy of
-    // this code.
+    // ===== softmax / correction / epilogue: thread = one query row
     setmaxnreg_inc<kRegsSoftmax>();
-    const int t = warp >> 2;        // stream of this warpgroup; it processes key steps h = t, t+2, ...
-    const int q = warp & 3;         // TMEM lane quarter this warp may touch
+    const int q = warp;             // TMEM lane quarter this warp may touch
     const int row = q * 32 + lane;  // row inside the 128-row query tile
     const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
-    const uint32_t o_addr = lane_addr + t * 128;
+    const uint32_t o_addr = lane_addr;
     const float c = p.scale_log2;
     float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
     const uint32_t my_bit = 1u << (row / B);  // query block of this row (uniform within a warp)
 #ifdef HEART_TRACE
-    const int tr0 = t ? 16 : 0;
-    const bool trw = (warp == 0 || warp == 4) && lane == 0;
+    const int tr0 = 0;
+    const bool trw = warp == 0 && lane == 0;
 #define HEART_TRS(slot)                   \
   do {                                    \
     if (trw) HEART_TR(h, tr0 + (slot));   \
@@ -402,8 +397,8 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   do {                  \
   } while (0)
 #endif
-    for (int h = t; h < NH && ok; h += 2) {
-      const int s = h & 3, ph = (h >> 2) & 1;
+    for (int h = 0; h < NH && ok; ++h) {
+      const int s = h % kStages, ph = (h / kStages) & 1;
       HEART_TRS(0);
       // key columns of this step that are real keys this row attends to
       int lim = 0;
@@ -412,7 +407,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         if ((e >> 16) & my_bit) lim = max(0, min(kStep, p.N - ((int)(e & 0xffff) * B + (h % HPB) * kStep)));
       }
       const int lim0 = min(lim, 32), lim1 = max(lim - 32, 0);
-      const uint32_t s_addr = lane_addr + 256 + s * kStep;
+      const uint32_t s_addr = lane_addr + 128 + s * kStep;
       ok = __all_sync(0xffffffffu, mbar_wait(&bars->qk_done[s], ph, abort));
       if (!ok) break;
       HEART_TRS(1);
@@ -448,9 +443,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
         m_ref = x_max;
         grow = true;
       }
-      if (__any_sync(0xffffffffu, grow) && h >= 2) {
-        // O_t must be quiescent: the previous product of this stream has to be complete
-        ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(h - 2) & 3], ((h - 2) >> 2) & 1, abort));
+      if (__any_sync(0xffffffffu, grow) && h >= 1) {
+        // O must be quiescent: the previous product has to be complete
+        ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(h - 1) % kStages], ((h - 1) / kStages) & 1, abort));
         if (!ok) break;
         tc_fence_after();
         const uint64_t alpha2 = pack_f32x2(alpha, alpha);
@@ -473,7 +468,7 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       HEART_TRS(4);
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       const uint64_t c2 = pack_f32x2(c, c), neg_m2 = pack_f32x2(neg_m, neg_m);
-      // p = 2^(s*c - m), packed to bf16 over columns [0, 32) of S[h & 3]; the product reads all 64
+      // p = 2^(s*c - m), packed to bf16 over columns [0, 32) of S[h & 1]; the product reads all 64
       // keys of the step, so every column is written (zeros where the row has no key)
       float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
@@ -512,55 +507,40 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
       if (lane == 0) HEART_TR(h, 24 + q);  // arrival time of each warp of the warpgroup
 #endif
     }
-    // epilogue: the two warpgroups exchange (max, sum) of their streams; warpgroup t then writes
-    // output dims [64t, 64t+64) of every row from both accumulators
-    const int n0 = (NH + 1) >> 1, n1 = NH >> 1;  // key steps per stream
+    // epilogue: O / l, one row per thread
     const int tok = row0 + row;
     const bool valid_row = tok < p.N;
-    xch[t * 256 + row] = m_ref;
-    xch[t * 256 + 128 + row] = l_run;
-    asm volatile("bar.sync 1, 256;" ::: "memory");  // the eight softmax warps (every one gets here)
-    ok = ok && !*abort;
-    const float m0 = xch[row], l0 = xch[128 + row], m1 = xch[256 + row], l1 = xch[384 + row];
-    // the products complete in issue order: the last one covers both streams
-    if (ok && NH > 0) ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(NH - 1) & 3], ((NH - 1) >> 2) & 1, abort));
+    // the products complete in issue order: the last one covers them all
+    if (ok && NH > 0)
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->pv_done[(NH - 1) % kStages], ((NH - 1) / kStages) & 1, abort));
     if (ok) {
       tc_fence_after();
-      const float m = fmaxf(m0, m1);
-      const float w0 = (n0 > 0 && m0 > -INFINITY) ? ex2(m0 - m) : 0.f;
-      const float w1 = (n1 > 0 && m1 > -INFINITY) ? ex2(m1 - m) : 0.f;
-      const float l = l0 * w0 + l1 * w1;
-      const float inv = l > 0.f ? 1.f / l : 0.f;
-      const float f0 = w0 * inv, f1 = w1 * inv;
-      uint16_t *orow = p.O + (long long)bidx * p.sb + (long long)hidx * p.sh + (long long)tok * p.sn + t * 64;
-      const uint32_t o_base = lane_addr + t * 64;
+      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+      uint16_t *orow = p.O + (long long)bidx * p.sb + (long long)hidx * p.sh + (long long)tok * p.sn;
 #pragma unroll 1
-      for (int ch = 0; ch < 4; ++ch) {  // 16 output dims at a time
-        uint32_t v0[16], v1[16];
-        if (n0 > 0) tmem_ld16(o_base + ch * 16, v0);
-        if (n1 > 0) tmem_ld16(o_base + 128 + ch * 16, v1);
-        tmem_wait_ld();
-        float o[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          o[i] = 0.f;
-          if (n0 > 0) o[i] = __uint_as_float(v0[i]) * f0;
-          if (n1 > 0) o[i] = fmaf(__uint_as_float(v1[i]), f1, o[i]);
+      for (int ch = 0; ch < 4; ++ch) {  // 32 output dims at a time
+        uint32_t v[32];
+        if (NH > 0) {
+          tmem_ld32(o_addr + ch * 32, v);
+          tmem_wait_ld();
         }
         if (valid_row) {
 #pragma unroll
-          for (int g4 = 0; g4 < 2; ++g4) {
+          for (int g4 = 0; g4 < 4; ++g4) {
+            float o[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[i] = NH > 0 ? __uint_as_float(v[g4 * 8 + i]) * inv : 0.f;
             uint4 w;
-            w.x = pack_bf16x2(o[g4 * 8 + 0], o[g4 * 8 + 1]);
-            w.y = pack_bf16x2(o[g4 * 8 + 2], o[g4 * 8 + 3]);
-            w.z = pack_bf16x2(o[g4 * 8 + 4], o[g4 * 8 + 5]);
-            w.w = pack_bf16x2(o[g4 * 8 + 6], o[g4 * 8 + 7]);
-            *reinterpret_cast<uint4 *>(orow + ch * 16 + g4 * 8) = w;
+            w.x = pack_bf16x2(o[0], o[1]);
+            w.y = pack_bf16x2(o[2], o[3]);
+            w.z = pack_bf16x2(o[4], o[5]);
+            w.w = pack_bf16x2(o[6], o[7]);
+            *reinterpret_cast<uint4 *>(orow + ch * 32 + g4 * 8) = w;
           }
         }
       }
-      if (t == 0 && valid_row && p.lse != nullptr)
-        p.lse[(size_t)r * p.N + tok] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      if (valid_row && p.lse != nullptr)
+        p.lse[(size_t)r * p.N + tok] = l_run > 0.f ? (m_ref + log2f(l_run)) * 0.6931471805599453f : -INFINITY;
     }
   }
 
@@ -569,9 +549,9 @@ __global__ void __launch_bounds__(kAttnThreads, 1)
   tc_fence_before();
   __syncthreads();
   if (tid == 0) HEART_TR(62, 3);
-  if (warp == kWarpQK0) {
+  if (warp == kWarpQK) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, kTmemCols);
   }
   if (tid == 0 && bars->abort) atomicExch(p.status, HEART_ERR_DEVICE_CHECK);
 }
@@ -614,6 +594,9 @@ cudaError_t launch_bk(const Geom &g, const CUtensorMap &mq, const CUtensorMap &m
                       const AttnParams &prm, cudaStream_t s) {
   const int smem = AttnSmem<B>::TOTAL + 1024;
   cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  // two CTAs per SM: all of the configurable shared memory
+  e = cudaFuncSetAttribute(attn_tc_kernel<B>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
   if (e != cudaSuccess) return e;
   attn_tc_kernel<B><<<g.B * prm.hcount * prm.n_ctas_per_head, kAttnThreads, smem, s>>>(mq, mk, mv, prm);
   return cudaGetLastError();
