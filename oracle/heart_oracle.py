@@ -228,3 +228,36 @@ def mask_iou(mask_a, mask_b, nb):
     counts = np.empty((R, 2), np.int64)
     lib().oracle_mask_iou(_p(mask_a), _p(mask_b), R, int(nb), _p(iou), _p(counts))
     return iou, counts
+
+
+# ---------------------------------------------------------------------------
+# Frequency-aware velocity error of the offline calibration (Eq. calibration error; appendix
+# "Frequency-aware velocity error"): 3-D DFT over (t, y, x) of every channel, fftshift, a frequency
+# is low along an axis of length n when it lies within floor(n/4) of the zero-frequency centre;
+# LL = low t, low y and low x; LH = low t, high on at least one spatial axis; HL = high t, low on
+# both spatial axes; HH = the rest.  Written straight from that definition with numpy's FFT.
+# ---------------------------------------------------------------------------
+BAND_WEIGHTS = (1.0, 0.5, 0.01, 0.01)  # (LL, LH, HL, HH)
+BAND_EPS = 1e-10
+
+
+def low_frequency_mask(n):
+    """Boolean mask over the fftshift-ed frequency index of an axis of length n."""
+    idx = np.arange(n)
+    return np.abs(idx - n // 2) <= n // 4
+
+
+def band_error(y_sparse, y_dense, weights=BAND_WEIGHTS, eps=BAND_EPS):
+    """y_*: [C, T, H, W].  Returns (e, band energies [LL, LH, HL, HH], denominator)."""
+    ys = np.asarray(y_sparse, np.float64)
+    yd = np.asarray(y_dense, np.float64)
+    err = ys - yd
+    E = np.fft.fftshift(np.fft.fftn(err, axes=(1, 2, 3)), axes=(1, 2, 3))
+    Y = np.fft.fftn(yd, axes=(1, 2, 3))
+    _, T, H, W = err.shape
+    lt = low_frequency_mask(T)[:, None, None]
+    ls = low_frequency_mask(H)[None, :, None] & low_frequency_mask(W)[None, None, :]
+    p = (E.real ** 2 + E.imag ** 2).sum(axis=0)
+    bands = np.array([p[lt & ls].sum(), p[lt & ~ls].sum(), p[~lt & ls].sum(), p[~lt & ~ls].sum()])
+    denom = float((Y.real ** 2 + Y.imag ** 2).sum() + eps)
+    return float(np.dot(np.asarray(weights, np.float64), bands) / denom), bands, denom

@@ -607,3 +607,79 @@ def test_full_token_drift_bounds_the_interaction_change(oracle):
     for r in range(R):
         delta_qk = np.abs((qa[r] + inc[r]) @ k[r].T - qa[r] @ k[r].T).mean() / math.sqrt(D)
         assert np.isclose(delta_qk, 2.0 / math.sqrt(D) * d[r], rtol=1e-13)
+
+
+# ----------------------------------------------------------------------------- calibration error
+def _brute_dft3(x):
+    """Direct O(n^2) 3-D DFT of one [T, H, W] array (separable, from the definition of the DFT)."""
+    out = x.astype(np.complex128)
+    for ax in range(3):
+        n = out.shape[ax]
+        k = np.arange(n)
+        F = np.exp(-2j * np.pi * np.outer(k, k) / n)
+        out = np.moveaxis(np.tensordot(F, np.moveaxis(out, ax, 0), axes=(1, 0)), 0, ax)
+    return out
+
+
+def test_band_error_against_direct_dft_and_parseval(oracle):
+    rs = np.random.RandomState(31)
+    C, T, H, W = 2, 5, 6, 9
+    yd = rs.standard_normal((C, T, H, W))
+    ys = yd + 0.1 * rs.standard_normal((C, T, H, W))
+    e, bands, denom = oracle.band_error(ys, yd)
+    # Parseval: the four bands partition the spectrum
+    assert np.isclose(bands.sum(), T * H * W * ((ys - yd) ** 2).sum(), rtol=1e-12)
+    assert np.isclose(denom, T * H * W * (yd ** 2).sum() + 1e-10, rtol=1e-12)
+    # band membership spelled out per unshifted frequency index: k is low iff min(k, n-k) <= n//4
+    # (the fftshift-ed distance to the centre n//2 is k for k < ceil(n/2) and n-k above, which for
+    # even n makes the Nyquist index n/2 lie at distance n/2)
+    def low(n):
+        k = np.arange(n)
+        return np.minimum(k, n - k) <= n // 4
+    lt, lh, lw = low(T), low(H), low(W)
+    ref = np.zeros(4)
+    for c in range(C):
+        P = np.abs(_brute_dft3(ys[c] - yd[c])) ** 2
+        for t in range(T):
+            for h in range(H):
+                for w in range(W):
+                    q = (0 if lt[t] else 2) + (0 if (lh[h] and lw[w]) else 1)
+                    ref[q] += P[t, h, w]
+    assert np.allclose(bands, ref, rtol=1e-10)
+    assert np.isclose(e, (1.0 * ref[0] + 0.5 * ref[1] + 0.01 * ref[2] + 0.01 * ref[3]) / denom, rtol=1e-10)
+
+
+@pytest.mark.parametrize("n,expected_low", [
+    (8, [0, 1, 2, 6, 7]),          # floor(8/4) = 2: |k| <= 2
+    (9, [0, 1, 2, 7, 8]),          # floor(9/4) = 2
+    (21, [0, 1, 2, 3, 4, 5, 16, 17, 18, 19, 20]),  # floor(21/4) = 5
+    (4, [0, 1, 3]),
+    (3, [0]),                      # floor(3/4) = 0: only the zero frequency
+])
+def test_band_low_frequency_rule(oracle, n, expected_low):
+    m = np.fft.ifftshift(oracle.low_frequency_mask(n))  # back to the unshifted index
+    assert sorted(np.nonzero(m)[0].tolist()) == expected_low
+
+
+def test_band_error_single_frequencies_and_weights(oracle):
+    C, T, H, W = 1, 8, 8, 12
+    t, h, w = np.meshgrid(np.arange(T), np.arange(H), np.arange(W), indexing="ij")
+    yd = np.ones((C, T, H, W))
+    N = T * H * W
+
+    def wave(kt, kh, kw):
+        return np.cos(2 * np.pi * (kt * t / T + kh * h / H + kw * w / W))[None]
+
+    # (kt, kh, kw) -> band; thresholds: T,H: |k| <= 2 low; W: |k| <= 3 low
+    for (kt, kh, kw), band in [((0, 0, 0), 0), ((2, 2, 3), 0), ((1, 3, 0), 1), ((2, 0, 4), 1),
+                               ((3, 1, 1), 2), ((4, 2, 3), 2), ((3, 3, 0), 3), ((4, 0, 6), 3)]:
+        e, bands, denom = oracle.band_error(yd + wave(kt, kh, kw), yd)
+        assert np.argmax(bands) == band and np.isclose(bands[band], bands.sum(), rtol=1e-12)
+        energy = N * (wave(kt, kh, kw) ** 2).sum()
+        assert np.isclose(e, oracle.BAND_WEIGHTS[band] * energy / (N * N + 1e-10), rtol=1e-12)
+    # homogeneity in the error, and the stabiliser when the reference is zero
+    e1, _, _ = oracle.band_error(yd + 0.5 * wave(1, 0, 0), yd)
+    e2, _, _ = oracle.band_error(yd + 1.5 * wave(1, 0, 0), yd)
+    assert np.isclose(e2, 9 * e1, rtol=1e-12)
+    e0, bands0, denom0 = oracle.band_error(wave(0, 0, 0) * 1e-3, np.zeros((C, T, H, W)))
+    assert denom0 == 1e-10 and np.isclose(e0, bands0[0] / 1e-10)
