@@ -200,6 +200,23 @@ int heart_full_token_drift(const heart_config *cfg, const void *Qa, const void *
 int heart_mask_iou(const heart_config *cfg, const uint32_t *mask_a, const uint32_t *mask_b,
                    double *iou_out, int64_t *counts_out, heart_stream_t stream);
 
+/* Frequency-aware velocity error of the offline calibration -- Eq. calibration error and the
+ * appendix paragraph "Frequency-aware velocity error" (an offline quantity: not on the layer-step path).
+ *   err = y_sparse - y_dense;  3-D DFT over (t, y, x) of every channel;  along an axis of length n a
+ *   frequency is low when it lies within floor(n/4) of the zero frequency (after fftshift);
+ *   LL = low t, low y and low x;  LH = low t, high on at least one spatial axis;
+ *   HL = high t, low on both spatial axes;  HH = the rest;
+ *   e = sum_q w_q * (spectral energy of err in band q) / (spectral energy of y_dense + eps).
+ * y_sparse, y_dense: fp32 [C, T, H, W], contiguous, device.  weights: host, (w_LL, w_LH, w_HL, w_HH)
+ * (the paper uses 1.0, 0.5, 0.01, 0.01 and eps = 1e-10).  out: device, fp64 [6] =
+ * (e, E_LL, E_LH, E_HL, E_HH, denominator), energies of the unnormalised DFT, summed over channels.
+ * workspace: heart_band_error_workspace_bytes(C, T, H, W) bytes of device scratch (four fp64 copies of
+ * the tensor), 256-byte aligned; it need not be cleared. */
+size_t heart_band_error_workspace_bytes(int32_t C, int32_t T, int32_t H, int32_t W);
+int heart_band_error(const float *y_sparse, const float *y_dense, int32_t C, int32_t T, int32_t H, int32_t W,
+                     const double *weights /* host [4] */, double eps, double *out, void *workspace,
+                     heart_stream_t stream);
+
 /* Synchronises `stream`, reads the workspace status word into *code_out (host) and clears it.
  * The only call that blocks. */
 int heart_get_status(void *workspace, heart_stream_t stream, int32_t *code_out /* host */);

@@ -93,4 +93,8 @@ int token_drift_chunks(const Geom &g, int *rows_per_cta);
 cudaError_t launch_mask_iou(const Geom &g, const uint32_t *A, const uint32_t *B, double *iou,
                             long long *counts, cudaStream_t s, int *launches);
 
+size_t band_error_workspace_bytes(int C, int T, int H, int W);
+cudaError_t launch_band_error(const float *ys, const float *yd, int C, int T, int H, int W, const double *weights,
+                              double eps, double *out, void *workspace, cudaStream_t s, int *launches);
+
 }  // namespace heart

@@ -330,6 +330,23 @@ int heart_mask_iou(const heart_config *cfg, const uint32_t *mask_a, const uint32
   return HEART_OK;
 }
 
+size_t heart_band_error_workspace_bytes(int32_t C, int32_t T, int32_t H, int32_t W) {
+  if (C < 1 || T < 1 || H < 1 || W < 1 || (long long)C * T * H * W > (1LL << 31)) return 0;
+  return band_error_workspace_bytes(C, T, H, W);
+}
+
+int heart_band_error(const float *y_sparse, const float *y_dense, int32_t C, int32_t T, int32_t H, int32_t W,
+                     const double *weights, double eps, double *out, void *workspace, heart_stream_t stream) {
+  if (heart_band_error_workspace_bytes(C, T, H, W) == 0) return HEART_ERR_INVALID;
+  if (!y_sparse || !y_dense || !weights || !out || !workspace || !(eps >= 0.0)) return HEART_ERR_INVALID;
+  if (reinterpret_cast<uintptr_t>(workspace) & 255u) return HEART_ERR_INVALID;
+  g_launches = 0;
+  cudaError_t e = launch_band_error(y_sparse, y_dense, C, T, H, W, weights, eps, out, workspace,
+                                    static_cast<cudaStream_t>(stream), &g_launches);
+  if (e != cudaSuccess) return cuda_fail(e, "band_error");
+  return HEART_OK;
+}
+
 int heart_get_status(void *workspace, heart_stream_t stream, int32_t *code_out) {
   if (!workspace || !code_out) return HEART_ERR_INVALID;
   cudaStream_t s = static_cast<cudaStream_t>(stream);

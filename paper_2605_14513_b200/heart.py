@@ -24,6 +24,7 @@ SYMBOLS = (
     "heart_workspace_bytes", "heart_state_reset", "heart_drift", "heart_predict_mask",
     "heart_block_sparse_attn", "heart_step", "heart_step_host", "heart_get_status", "heart_strerror",
     "heart_last_launch_count", "heart_drift_static", "heart_full_token_drift", "heart_mask_iou",
+    "heart_band_error_workspace_bytes", "heart_band_error",
 )
 
 
@@ -76,6 +77,10 @@ def lib():
         l.heart_full_token_drift.restype = C.c_int
         l.heart_mask_iou.argtypes = [C.POINTER(Config)] + [vp] * 5
         l.heart_mask_iou.restype = C.c_int
+        l.heart_band_error_workspace_bytes.argtypes = [C.c_int32] * 4
+        l.heart_band_error_workspace_bytes.restype = C.c_size_t
+        l.heart_band_error.argtypes = [vp, vp] + [C.c_int32] * 4 + [C.POINTER(C.c_double), C.c_double, vp, vp, vp]
+        l.heart_band_error.restype = C.c_int
         for fn in ("heart_state_reset", "heart_drift", "heart_predict_mask", "heart_block_sparse_attn",
                    "heart_step", "heart_step_host", "heart_get_status"):
             getattr(l, fn).restype = C.c_int
@@ -204,6 +209,23 @@ def heart_mask_iou(cfg, mask_a, mask_b, iou_out, counts_out=None):
     counts_out: optional int64 [R, 2] = (intersection, union)."""
     _check(lib().heart_mask_iou(C.byref(cfg), _ptr(mask_a), _ptr(mask_b), _ptr(iou_out), _ptr(counts_out),
                                 _stream()))
+
+
+def heart_band_error(y_sparse, y_dense, weights=(1.0, 0.5, 0.01, 0.01), eps=1e-10):
+    """Four-band 3-D DFT calibration error of y_sparse against y_dense (fp32 [C, T, H, W] on the GPU).
+    Returns a device tensor of 6 doubles: (e, E_LL, E_LH, E_HL, E_HH, denominator)."""
+    assert y_sparse.dtype == torch.float32 and y_dense.dtype == torch.float32
+    assert y_sparse.is_contiguous() and y_dense.is_contiguous() and y_sparse.shape == y_dense.shape
+    Cc, T, H, W = y_sparse.shape
+    nbytes = lib().heart_band_error_workspace_bytes(Cc, T, H, W)
+    if nbytes == 0:
+        raise HeartError(ERR_INVALID)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=y_sparse.device)
+    out = torch.empty(6, dtype=torch.float64, device=y_sparse.device)
+    w = (C.c_double * 4)(*weights)
+    _check(lib().heart_band_error(_ptr(y_sparse), _ptr(y_dense), Cc, T, H, W, w, float(eps), _ptr(out), _ptr(ws),
+                                  _stream()))
+    return out
 
 
 def heart_get_status(ws) -> int:

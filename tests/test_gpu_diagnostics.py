@@ -128,3 +128,49 @@ def test_mask_iou_random_bits_at_maximum_size(heart, oracle):
     heart.heart_mask_iou(cfg, ta, tb, iou, counts)
     iou_o, counts_o = oracle.mask_iou(a, b, nb)
     assert np.array_equal(to_np(counts), counts_o) and np.array_equal(to_np(iou), iou_o)
+
+
+# ----------------------------------------------------------------------------- calibration error
+@pytest.mark.parametrize("shape", [
+    (2, 5, 6, 9),        # odd and even axes, tiny
+    (1, 8, 8, 12),       # the single-frequency grid of the oracle pins
+    (3, 7, 20, 33),      # several thousand elements per channel
+    (16, 21, 30, 52),    # a 480P latent at half resolution: 524k elements
+])
+def test_band_error_matches_oracle(heart, oracle, shape):
+    gen = torch.Generator(device="cuda").manual_seed(sum(shape))
+    yd = torch.randn(shape, device="cuda", generator=gen)
+    # error with structure in every band: smooth part + white noise
+    C, T, H, W = shape
+    t = torch.arange(T, device="cuda").view(1, T, 1, 1) / T
+    h = torch.arange(H, device="cuda").view(1, 1, H, 1) / H
+    smooth = 0.3 * torch.cos(2 * np.pi * (t + h))
+    ys = (yd + smooth + 0.05 * torch.randn(shape, device="cuda", generator=gen)).contiguous()
+    out = to_np(heart.heart_band_error(ys, yd))
+    e, bands, denom = oracle.band_error(to_np(ys), to_np(yd))
+    total = bands.sum()
+    assert np.allclose(out[1:5], bands, rtol=1e-9, atol=1e-12 * total)
+    assert np.isclose(out[5], denom, rtol=1e-12)
+    assert np.isclose(out[0], e, rtol=1e-9)
+    # run to run bit-reproducible
+    assert np.array_equal(to_np(heart.heart_band_error(ys, yd)), out)
+
+
+def test_band_error_single_frequencies_on_gpu(heart, oracle):
+    C, T, H, W = 1, 8, 8, 12
+    t, h, w = np.meshgrid(np.arange(T), np.arange(H), np.arange(W), indexing="ij")
+    yd = torch.ones((C, T, H, W), device="cuda")
+    for (kt, kh, kw), band in [((0, 0, 0), 0), ((2, 2, 3), 0), ((1, 3, 0), 1), ((2, 0, 4), 1), ((3, 1, 1), 2),
+                               ((4, 2, 3), 2), ((3, 3, 0), 3), ((4, 0, 6), 3)]:
+        wave = np.cos(2 * np.pi * (kt * t / T + kh * h / H + kw * w / W))[None].astype(np.float32)
+        ys = yd + torch.from_numpy(wave).cuda()
+        out = to_np(heart.heart_band_error(ys.contiguous(), yd))
+        e, bands, _ = oracle.band_error(to_np(ys), to_np(yd))
+        assert int(np.argmax(out[1:5])) == band
+        assert np.allclose(out[1:5], bands, rtol=1e-9, atol=1e-9 * bands.sum()) and np.isclose(out[0], e, rtol=1e-9)
+    # identical tensors: zero error; zero reference: the stabiliser alone in the denominator
+    out = to_np(heart.heart_band_error(yd, yd))
+    assert np.all(out[:5] == 0)
+    z = torch.zeros_like(yd)
+    out = to_np(heart.heart_band_error(yd * 1e-3, z))
+    assert out[5] == 1e-10
