@@ -79,10 +79,16 @@ typedef struct {
   int32_t *kv_cnt;             /* [R, n_b] number of retained key blocks per query block   */
 } heart_state;
 
-/* Bytes of scratch every compute call needs (block sums, means, flags, status
- * word).  Host-only; returns 0 for an invalid or unsupported config.  The caller
- * allocates it once (256-byte aligned) and zero-fills it before first use. */
+/* Bytes of scratch every compute call needs (block means, token means, flags, status
+ * word, and the pooled scores of the mask predictor: 8 * R * n_b * roundup(n_b, 32) bytes,
+ * by far the largest part).  Host-only; returns 0 for an invalid or unsupported config.
+ * The caller allocates it once (256-byte aligned) and zero-fills it before first use. */
 size_t heart_workspace_bytes(const heart_config *cfg /* host */);
+
+/* The leading part of that workspace which heart_drift alone reads and writes (everything
+ * but the pooled scores).  A caller that only ever calls heart_drift may allocate just this
+ * much.  Host-only; 0 for an invalid or unsupported config. */
+size_t heart_drift_workspace_bytes(const heart_config *cfg /* host */);
 
 /* Clears has_anchor (and zeroes kv_cnt) so the next step refreshes every head
  * (Algorithm 1, "no cached anchor exists"). */
@@ -95,7 +101,7 @@ int heart_state_reset(const heart_config *cfg, heart_state *st /* host struct */
  *                 fraction < gate_lo -> anchored heads reuse, fraction > gate_hi -> all refresh);
  *   refreshed heads: anchor <- current means, has_anchor <- 1.
  * delta [R] fp64 (a negative entry always refreshes).  drift_out [R] fp64 and refresh_out [R] u8
- * may each be NULL.  Also leaves the per-block sums of Q and K in the workspace. */
+ * may each be NULL.  Also leaves the per-block means of Q and K in the workspace. */
 int heart_drift(const heart_config *cfg, const void *Q, const void *K, const double *delta,
                 heart_state *st, double *drift_out, uint8_t *refresh_out, void *workspace,
                 heart_stream_t stream);
@@ -160,15 +166,15 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
  * allocator-managed region where foreign allocations are forbidden or would fragment a fully
  * reserved GPU, in a real-time or callback context that must not block on the driver's allocator,
  * or a plugin that is handed Q/K and the TMR state but no way to obtain scratch.  Such a caller
- * still passes its inputs, outputs and state; only the scratch (block sums, means, flags) comes
+ * still passes its inputs, outputs and state; only the scratch (block means, token means, flags) comes
  * from a fixed HEART_STATIC_SCRATCH_BYTES array compiled into the library.  The call makes no
  * cudaMalloc / cudaFree and calls no allocating routine.
  *
  * Same arguments, results and error codes as heart_drift, except:
  *   - no `workspace`; st->mask_bits / kv_idx / kv_cnt may be NULL (they are not touched);
- *   - a shape whose heart_workspace_bytes exceeds HEART_STATIC_SCRATCH_BYTES is rejected with
+ *   - a shape whose heart_drift_workspace_bytes exceeds HEART_STATIC_SCRATCH_BYTES is rejected with
  *     HEART_ERR_TOO_LARGE before anything is launched;
- *   - the per-block sums it leaves behind are in the built-in array, not in a caller workspace,
+ *   - the per-block means it leaves behind are in the built-in array, not in a caller workspace,
  *     so a following heart_predict_mask recomputes them (it always does).
  * The array is part of the library image: every GPU that loads the library holds those 16 MiB
  * until the process exits.  The first call on each device looks the array's device address up

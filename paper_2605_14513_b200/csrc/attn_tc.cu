@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
 #endif
 
   // ------------------------------------------------------------------ set-up
-  if (tid == 0) HEART_TR(62, 0);
+  if (tid == 0) HEART_TR(0, 28);
   // The lists of this tile's query blocks come from global memory: their loads are issued first
   // (speculatively, inside the row pitch) so that their latency overlaps the rest of the set-up.
   constexpr int kPre = kMaxNb / kAttnThreads;  // entries per thread held in registers
@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (tid == 0) HEART_TR(62, 1);
+  if (tid == 0) HEART_TR(0, 29);
   const uint32_t tmem = bars->tmem_base;
   const int U = bars->n_union;
   const int NH = U * HPB;  // key steps; step h uses S buffer and shared-memory stage h & 1
@@ -545,10 +545,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
   }
 
   // ------------------------------------------------------------------ tear-down
-  if (tid == 0) HEART_TR(62, 2);
+  if (tid == 0) HEART_TR(0, 30);
   tc_fence_before();
   __syncthreads();
-  if (tid == 0) HEART_TR(62, 3);
+  if (tid == 0) HEART_TR(0, 31);
   if (warp == kWarpQK) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);

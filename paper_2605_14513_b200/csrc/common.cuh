@@ -36,13 +36,15 @@ __host__ inline void set_chunks(Geom &g) {
 struct Workspace {
   int32_t *status;    // [64]   word 0: sticky device-check code; word 1: detail; word 8: ticket counter
                       //        of the drift kernel (zero between launches)
-  double *bsum;       // [2][R][nb][D]  per-block sums of Q (0) and K (1)
+  double *bmean;      // [2][R][nb][D]  per-block (pooled) means of Q (0) and K (1)
   double *psum;       // [2][R][nchunks][D]  per-CTA partial token sums
   double *mean;       // [2][R][D]      token means of the current step
   double *part;       // [2][R]         L1 parts of the drift
   uint8_t *pre;       // [R]            head-wise decision before the gate
   uint8_t *refresh;   // [R]            final decision of the current step
   double *drift;      // [R]
+  double *scores;     // [R][nb][pitch] pooled scores of the refreshed heads, pitch = nb rounded up to 32
+  size_t bytes_drift;  // what heart_drift alone touches (everything above `scores`)
   size_t bytes;
 };
 
@@ -54,7 +56,7 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   size_t off = 0;
   w.status = reinterpret_cast<int32_t *>(p + off);
   off += align256(64 * sizeof(int32_t));
-  w.bsum = reinterpret_cast<double *>(p + off);
+  w.bmean = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * 2 * (size_t)g.R * g.nb * kD);
   w.psum = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * 2 * (size_t)g.R * g.nchunks * kD);
@@ -68,6 +70,9 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   off += align256((size_t)g.R);
   w.drift = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * (size_t)g.R);
+  w.bytes_drift = off;
+  w.scores = reinterpret_cast<double *>(p + off);
+  off += align256(sizeof(double) * (size_t)g.R * g.nb * (size_t)(((g.nb + 31) / 32) * 32));
   w.bytes = off;
   return w;
 }

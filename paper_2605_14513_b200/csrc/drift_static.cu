@@ -42,8 +42,9 @@ extern "C" {
 int heart_drift_static(const heart_config *cfg, const void *Q, const void *K, const double *delta,
                        heart_state *st, double *drift_out, uint8_t *refresh_out, heart_stream_t stream) {
   if (cfg == nullptr) return HEART_ERR_INVALID;
-  // Size check first, from the same accounting the caller-allocated path uses.
-  const size_t need = heart_workspace_bytes(cfg);
+  // Size check first, from the same accounting the caller-allocated path uses (the part of the
+  // workspace that the drift kernels touch: the pooled-score area of the mask predictor lies behind it).
+  const size_t need = heart_drift_workspace_bytes(cfg);
   if (need == 0) return HEART_ERR_UNSUPPORTED;  // shape the library does not handle at all
   if (need > (size_t)HEART_STATIC_SCRATCH_BYTES) return HEART_ERR_TOO_LARGE;
   if (!Q || !K || !delta || !st || !st->anchor_q || !st->anchor_k || !st->has_anchor) return HEART_ERR_INVALID;

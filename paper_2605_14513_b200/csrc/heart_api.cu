@@ -81,6 +81,12 @@ size_t heart_workspace_bytes(const heart_config *cfg) {
   return carve(g, nullptr).bytes;
 }
 
+size_t heart_drift_workspace_bytes(const heart_config *cfg) {
+  Geom g;
+  if (make_geom(cfg, &g) != HEART_OK) return 0;
+  return carve(g, nullptr).bytes_drift;
+}
+
 int heart_state_reset(const heart_config *cfg, heart_state *st, heart_stream_t stream) {
   Geom g;
   int rc = make_geom(cfg, &g);
@@ -311,7 +317,7 @@ int heart_full_token_drift(const heart_config *cfg, const void *Qa, const void *
   const size_t need = (size_t)g.R * token_drift_chunks(g, &rows);  // partials live in the block-sum area
   if (need > 2 * (size_t)g.R * g.nb * kD) return HEART_ERR_INVALID;
   g_launches = 0;
-  cudaError_t e = launch_token_drift(g, Qa, Ka, Qb, Kb, w.bsum, drift_out,
+  cudaError_t e = launch_token_drift(g, Qa, Ka, Qb, Kb, w.bmean, drift_out,
                                      static_cast<cudaStream_t>(stream), &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "token_drift");
   return HEART_OK;

@@ -2,27 +2,27 @@
 // importance, retain until the accumulated importance reaches the head's threshold; the minimal
 // cumulative-mass set of Observation I).  Importance = row softmax of the block-pooled Q.K^T scores.
 //
-// One CTA owns TI = 16 query blocks of one head.  Phase 1 is a register-tiled fp64 contraction of
-// the pooled means (each thread 8 query blocks x 4 key blocks, key means staged through shared
-// memory 512 blocks x 16 dims at a time with the next stage's loads in flight) into a shared-memory
-// tile of scores.  Phase 2 gives each
-// warp two rows: two-pass softmax, then top-p WITHOUT a sort: the kept set is {p > theta} plus the
-// lowest-index ties at theta, where theta is the largest element value whose ">= theta" mass still
-// reaches tau -- found by a search over the IEEE-754 pattern of p (positive doubles order like
-// their bit patterns): the top 14 bits two at a time over all blocks, the rest directly over the
-// few blocks that share that prefix.  Everything is fp64 so the integer outputs (bit mask,
-// ascending index list, count) agree with a plain fp64 sort-and-accumulate reference except when
-// the cumulative mass is within rounding (1e-15) of tau.
-#include <type_traits>
-
+// Two kernels.  pooled_scores_kernel is a register-tiled fp64 contraction of the pooled means: a CTA
+// owns 64 query blocks x 128 key blocks of one head (each thread 8 x 4), the means arrive 16 dims at
+// a time by cp.async into a double-buffered shared-memory tile, and every score accumulates over the
+// 128 dims in ascending order in one fma chain.  The scores go to the workspace (they stay in L2).
+// top_p_kernel gives each warp one row: two-pass softmax, then top-p WITHOUT a sort: the kept set is
+// {p > theta} plus the lowest-index ties at theta, where theta is the largest element value whose
+// ">= theta" mass still reaches tau -- found by a search over the IEEE-754 pattern of p (positive
+// doubles order like their bit patterns): the top 14 bits two at a time over all blocks, the rest
+// directly over the few blocks that share that prefix.  Everything is fp64 so the integer outputs
+// (bit mask, ascending index list, count) agree with a plain fp64 sort-and-accumulate reference
+// except when the cumulative mass is within rounding (1e-15) of tau.
 #include "common.cuh"
 
 namespace heart {
 
-constexpr int TI = 16;    // query blocks per CTA
-constexpr int TJ = 512;   // key blocks per staged pass
+constexpr int SI = 64;    // query blocks per CTA of the score kernel
+constexpr int SJ = 128;   // key blocks per CTA
 constexpr int TD = 16;    // dims per staged chunk
 constexpr int KLD = TD + 1;
+constexpr int kRowsPerCta = 8;  // rows (warps) per CTA of the top-p kernel
+constexpr int kMaxCand = 64;    // candidates the direct threshold evaluation takes
 
 __device__ __forceinline__ double warp_sum(double v) {
 #pragma unroll
@@ -35,120 +35,112 @@ __device__ __forceinline__ double warp_max(double v) {
   return v;
 }
 
-template <int NJ>  // NJ*32 >= n_b
-__global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restrict__ bsum, int R, int N,
-                                                           int block, int nb, double scale,
-                                                           const double *__restrict__ tau,
-                                                           const uint8_t *__restrict__ refresh,
-                                                           unsigned flags, uint32_t *__restrict__ mask_bits,
-                                                           int32_t *__restrict__ kv_idx,
-                                                           int32_t *__restrict__ kv_cnt, int idx_stride,
-                                                           int W) {
-  constexpr int NBP = NJ * 32;
-  const int r = blockIdx.y;
-  if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: mask untouched
-  const int I0 = blockIdx.x * TI;
+// 8-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead
+__device__ __forceinline__ void cp_async8(double *smem_dst, const double *src, int src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
+               "l"(src), "r"(src_bytes)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+// scores[r][I][J] = scale * <mean_q[r][I], mean_k[r][J]> for the refreshed heads r.
+__global__ void __launch_bounds__(256, 2) pooled_scores_kernel(const double *__restrict__ bmean, int R, int nb,
+                                                               int pitch, double scale,
+                                                               const uint8_t *__restrict__ refresh,
+                                                               double *__restrict__ scores) {
+  const int r = blockIdx.z;
+  if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: nothing to predict
+  const int I0 = blockIdx.y * SI, J0 = blockIdx.x * SJ;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double *S = reinterpret_cast<double *>(smem_raw);  // [TI][NBP]
-  double *Qs = S + TI * NBP;                         // [TI][kD]
-  double *Ks = Qs + TI * kD;                         // [TJ][KLD]
-  const double *bq = bsum + ((size_t)r * nb) * kD;
-  const double *bk = bsum + (((size_t)R + r) * nb) * kD;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int last_cnt = N - (nb - 1) * block;
-  const double inv_block = 1.0 / (double)block;
-
-  for (int e = tid; e < TI * kD; e += 256) {
-    const int i = e / kD, I = I0 + i;
-    double v = 0.0;
-    if (I < nb) v = (I == nb - 1) ? bq[(size_t)I * kD + (e % kD)] / (double)last_cnt : bq[(size_t)I * kD + (e % kD)] * inv_block;
-    Qs[e] = v;
-  }
-
-  // ---- phase 1: S[i][J] = scale * <Qp[I0+i], Kp[J]>.  Each thread owns 8 query blocks x 4 key blocks;
-  // the key means are staged 512 blocks x 16 dims at a time, and the loads of the next stage are in
-  // flight (in registers) while the current one is multiplied.
-  const int rg = tid >> 7, cl = tid & 127;
-  constexpr int PER = (TJ * TD) / 256;  // staged values per thread = 32
-  const int n_jc = (nb + TJ - 1) / TJ, n_stage = n_jc * (kD / TD);
-  double pre[PER];
-  auto fetch = [&](int stage) {
-    const int jc = (stage / (kD / TD)) * TJ, dc = (stage % (kD / TD)) * TD;
+  double *tile = reinterpret_cast<double *>(smem_raw);  // [2][SI + SJ][KLD]: query rows, then key rows
+  const double *bq = bmean + ((size_t)r * nb) * kD;
+  const double *bk = bmean + (((size_t)R + r) * nb) * kD;
+  const int tid = threadIdx.x;
+  constexpr int kRows = SI + SJ, kPer = kRows * TD / 256;  // 12 copies per thread and stage
+  auto stage_in = [&](int stage, int buf) {
+    const int dc = stage * TD;
+    double *dst = tile + (size_t)buf * kRows * KLD;
 #pragma unroll
-    for (int k = 0; k < PER; ++k) {
-      const int e = tid + 256 * k, J = jc + e / TD;
-      pre[k] = (J < nb) ? bk[(size_t)J * kD + dc + (e % TD)] : 0.0;
+    for (int k = 0; k < kPer; ++k) {
+      const int e = tid + 256 * k, row = e / TD, dd = e % TD;
+      const int blk = row < SI ? I0 + row : J0 + row - SI;
+      const double *src = (row < SI ? bq : bk) + (size_t)min(blk, nb - 1) * kD + dc + dd;
+      cp_async8(dst + row * KLD + dd, src, blk < nb ? 8 : 0);
     }
+    cp_async_commit();
   };
-  fetch(0);
+  const int rg = tid >> 5, cl = tid & 31;  // rows rg*8 .. rg*8+7, key columns cl + 32 m
   double acc[8][4];
-  for (int stage = 0; stage < n_stage; ++stage) {
-    const int jc = (stage / (kD / TD)) * TJ, dc = (stage % (kD / TD)) * TD;
-    if (dc == 0) {
 #pragma unroll
-      for (int a = 0; a < 8; ++a)
+  for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int m = 0; m < 4; ++m) acc[a][m] = 0.0;
-    }
-    __syncthreads();  // the previous stage has been consumed
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-      const int e = tid + 256 * k, row = e / TD, J = jc + row;
-      // full blocks: 1/block is a power of two, so the product equals the division exactly
-      Ks[row * KLD + (e % TD)] = (J == nb - 1) ? pre[k] / (double)last_cnt : pre[k] * inv_block;
+    for (int m = 0; m < 4; ++m) acc[a][m] = 0.0;
+  stage_in(0, 0);
+  for (int stage = 0; stage < kD / TD; ++stage) {
+    const int buf = stage & 1;
+    if (stage + 1 < kD / TD) {
+      stage_in(stage + 1, buf ^ 1);  // its buffer was released by the barrier that ended stage - 1
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
     }
     __syncthreads();
-    if (stage + 1 < n_stage) fetch(stage + 1);
-    // column groups of 128 key blocks that exist in this pass (the last pass is usually short)
-    const int nm = min(4, (nb - jc + 127) >> 7);
-    auto multiply = [&](auto NM) {
-      constexpr int kNm = decltype(NM)::value;
+    const double *Qs = tile + (size_t)buf * kRows * KLD, *Ks = Qs + SI * KLD;
 #pragma unroll 4
-      for (int dd = 0; dd < TD; ++dd) {
-        double q[8], k4[kNm];
+    for (int dd = 0; dd < TD; ++dd) {
+      double q[8], k4[4];
 #pragma unroll
-        for (int a = 0; a < 8; ++a) q[a] = Qs[(rg * 8 + a) * kD + dc + dd];
+      for (int a = 0; a < 8; ++a) q[a] = Qs[(rg * 8 + a) * KLD + dd];
 #pragma unroll
-        for (int m = 0; m < kNm; ++m) k4[m] = Ks[(cl + 128 * m) * KLD + dd];
-#pragma unroll
-        for (int a = 0; a < 8; ++a)
-#pragma unroll
-          for (int m = 0; m < kNm; ++m) acc[a][m] = fma(q[a], k4[m], acc[a][m]);
-      }
-    };
-    if (nm == 4)
-      multiply(std::integral_constant<int, 4>{});
-    else if (nm == 3)
-      multiply(std::integral_constant<int, 3>{});
-    else if (nm == 2)
-      multiply(std::integral_constant<int, 2>{});
-    else
-      multiply(std::integral_constant<int, 1>{});
-    if (dc == kD - TD) {
+      for (int m = 0; m < 4; ++m) k4[m] = Ks[(cl + 32 * m) * KLD + dd];
 #pragma unroll
       for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int m = 0; m < 4; ++m) {
-          const int J = jc + cl + 128 * m;
-          if (J < NBP) S[(rg * 8 + a) * NBP + J] = acc[a][m] * scale;
-        }
+        for (int m = 0; m < 4; ++m) acc[a][m] = fma(q[a], k4[m], acc[a][m]);
+    }
+    __syncthreads();  // this stage's buffer may be refilled
+  }
+#pragma unroll
+  for (int a = 0; a < 8; ++a) {
+    const int I = I0 + rg * 8 + a;
+    if (I >= nb) continue;
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+      const int J = J0 + cl + 32 * m;
+      if (J < pitch) scores[((size_t)r * nb + I) * pitch + J] = acc[a][m] * scale;
     }
   }
-  __syncthreads();
+}
 
-  // ---- phase 2: per-row softmax and top-p; warp w owns rows 2w and 2w+1
+template <int NJ>  // NJ*32 >= n_b
+__global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *__restrict__ scores, int nb, int pitch,
+                                                                 const double *__restrict__ tau,
+                                                                 const uint8_t *__restrict__ refresh,
+                                                                 unsigned flags, uint32_t *__restrict__ mask_bits,
+                                                                 int32_t *__restrict__ kv_idx,
+                                                                 int32_t *__restrict__ kv_cnt, int idx_stride,
+                                                                 int W) {
+  const int r = blockIdx.y;
+  if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: mask untouched
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __shared__ double cand[kRowsPerCta][kMaxCand];
   const unsigned lt_mask = (1u << lane) - 1u;
-  for (int i = warp * 2; i < warp * 2 + 2; ++i) {
-    const int I = I0 + i;
-    if (I >= nb) continue;
+  {
+    const int I = blockIdx.x * kRowsPerCta + warp;
+    if (I >= nb) return;
     const size_t row = (size_t)r * nb + I;
+    const double *srow = scores + row * pitch;
     double p[NJ];
     const double neg_inf = __longlong_as_double(0xfff0000000000000LL);
     double mx = neg_inf;
 #pragma unroll
     for (int j = 0; j < NJ; ++j) {
       const int J = j * 32 + lane;
-      p[j] = (J < nb) ? S[i * NBP + J] : neg_inf;
+      p[j] = (J < nb) ? srow[J] : neg_inf;
       mx = fmax(mx, p[j]);
     }
     mx = warp_max(mx);
@@ -160,85 +152,90 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
       z += p[j];
     }
     z = warp_sum(z);
-    double total = 0.0;
-#pragma unroll
-    for (int j = 0; j < NJ; ++j) {
-      p[j] = p[j] / z;
-      total += p[j];
-    }
-    total = warp_sum(total);
-
-    const double t = (flags & HEART_FORCE_DENSE) ? 1.0 : tau[r];
-    const bool keep_all = !(t < 1.0) || !(total >= t);
+    // From here on p holds the unnormalised weights e = exp(s - max) <= 1 and every mass is compared
+    // with tau * z instead of dividing the row by z: the same ranking, the same ties and the same
+    // cumulative-mass test up to rounding, at 1/3 fewer fp64 instructions per block.
+    const double tau_r = (flags & HEART_FORCE_DENSE) ? 1.0 : tau[r];
+    const double t = tau_r * z;
+    const bool keep_all = !(tau_r < 1.0) || !(z >= t);
     long long theta = 0;
-    int m_ties = 0;
+    int m_ties = 0, n_ties = 0;
     if (!keep_all) {
-      // Full-width rounds for the exponent and the top mantissa bits ...
-      auto mass_at_least = [&](long long cand) -> double {
-        double g0 = 0.0, g1 = 0.0, g2 = 0.0, g3 = 0.0;  // fixed 4-way split: same order on every run
-#pragma unroll
-        for (int j = 0; j < NJ; j += 4) {
-          if (__double_as_longlong(p[j]) >= cand) g0 += p[j];
-          if (j + 1 < NJ && __double_as_longlong(p[j + 1]) >= cand) g1 += p[j + 1];
-          if (j + 2 < NJ && __double_as_longlong(p[j + 2]) >= cand) g2 += p[j + 2];
-          if (j + 3 < NJ && __double_as_longlong(p[j + 3]) >= cand) g3 += p[j + 3];
-        }
-        return warp_sum((g0 + g1) + (g2 + g3));
-      };
-      constexpr int kSplit = 48;  // bits [kSplit, 62) are searched over all blocks, two bits a round
-      // (three trial thresholds per round: their three reductions run side by side)
-      auto masses_at_least = [&](long long c1, long long c2, long long c3, double &m1, double &m2, double &m3) {
-        double a1 = 0.0, a2 = 0.0, a3 = 0.0, b1 = 0.0, b2 = 0.0, b3 = 0.0;  // fixed split: same order on every run
+      // Rounds over all blocks, two bits of theta each: three trial thresholds per round, their three
+      // reductions side by side (fixed split of the sums: same order on every run).
+      auto round2 = [&](int bit) {
+        // trial patterns theta | 01, 10, 11 at bits (bit+1, bit): the mass is non-increasing in them
+        // (bit >= 32: the low words of the patterns are zero, so comparing the high words decides)
+        const long long c1 = theta | (1LL << bit), c2 = theta | (2LL << bit), c3 = theta | (3LL << bit);
+        const int h1 = (int)(c1 >> 32), h2 = (int)(c2 >> 32), h3 = (int)(c3 >> 32);
+        double a1 = 0.0, a2 = 0.0, a3 = 0.0, b1 = 0.0, b2 = 0.0, b3 = 0.0;
 #pragma unroll
         for (int j = 0; j < NJ; j += 2) {
-          const long long k0 = __double_as_longlong(p[j]), k1 = __double_as_longlong(p[j + 1]);
-          if (k0 >= c1) a1 += p[j];
-          if (k0 >= c2) a2 += p[j];
-          if (k0 >= c3) a3 += p[j];
-          if (k1 >= c1) b1 += p[j + 1];
-          if (k1 >= c2) b2 += p[j + 1];
-          if (k1 >= c3) b3 += p[j + 1];
+          const int k0 = __double2hiint(p[j]), k1 = __double2hiint(p[j + 1]);
+          if (k0 >= h1) a1 += p[j];
+          if (k0 >= h2) a2 += p[j];
+          if (k0 >= h3) a3 += p[j];
+          if (k1 >= h1) b1 += p[j + 1];
+          if (k1 >= h2) b2 += p[j + 1];
+          if (k1 >= h3) b3 += p[j + 1];
         }
-        m1 = a1 + b1;
-        m2 = a2 + b2;
-        m3 = a3 + b3;
+        double m1 = a1 + b1, m2 = a2 + b2, m3 = a3 + b3;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
           m1 += __shfl_xor_sync(0xffffffffu, m1, o);
           m2 += __shfl_xor_sync(0xffffffffu, m2, o);
           m3 += __shfl_xor_sync(0xffffffffu, m3, o);
         }
-      };
-      static_assert((62 - kSplit) % 2 == 0 && NJ % 2 == 0, "two bits per round, two blocks per step");
-      for (int bit = 60; bit >= kSplit; bit -= 2) {
-        // trial patterns theta | 01, 10, 11 at bits (bit+1, bit): the mass is non-increasing in them
-        const long long c1 = theta | (1LL << bit), c2 = theta | (2LL << bit), c3 = theta | (3LL << bit);
-        double m1, m2, m3;
-        masses_at_least(c1, c2, c3, m1, m2, m3);
         theta = (m3 >= t) ? c3 : (m2 >= t) ? c2 : (m1 >= t) ? c1 : theta;
+      };
+      static_assert(NJ % 2 == 0, "two blocks per step");
+      // The exponent and the top four mantissa bits first (bits 61..48; bit 62 is clear for p <= 1) ...
+      constexpr int low = 48;  // bits [low, 62) of theta are decided over all blocks
+      static_assert(low >= 32, "the full-width rounds compare high words only");
+      // theta is the value of one of the blocks, so it shares the leading bits that the largest and
+      // the smallest weight of the row have in common: the rounds start below them.
+      int first_bit = 60;
+      {
+        int hmax = 0, hmin = 0x7fffffff;
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) {
+          const int h = __double2hiint(p[j]);
+          hmax = max(hmax, h);
+          if (j * 32 + lane < nb) hmin = min(hmin, h);
+        }
+        hmax = __reduce_max_sync(0xffffffffu, hmax);
+        hmin = __reduce_min_sync(0xffffffffu, hmin);
+        const int top = 63 - __clz(hmax ^ hmin);  // highest bit (of the 64) in which they differ; 31 if none in the high word
+        first_bit = min(60, top & ~1);            // the round at `bit` decides bits (bit + 1, bit)
+        if (first_bit + 2 < 62) theta = ((long long)hmax << 32) & ~((1LL << (first_bit + 2)) - 1);
       }
+      for (int bit = first_bit; bit >= low; bit -= 2) round2(bit);
+      if (first_bit < low) theta &= ~((1LL << low) - 1);  // the whole searched prefix is common
       // ... then only the blocks whose pattern shares that prefix can still decide the remaining bits:
-      // they are compacted (through this row's no longer needed score slots) and the other 48 rounds
-      // run on at most two candidates per lane.  Blocks above the prefix enter as one constant.
-      const long long hi = theta >> kSplit;
-      double *scr = S + i * NBP;
+      // they are compacted into shared memory (the first kMaxCand of them; more than that takes the
+      // slow path below, which does not read the list).  Blocks above the prefix enter as one constant.
+      const long long hi = theta >> low;
+      double *scr = cand[warp];
       double ab0 = 0.0, ab1 = 0.0;
       int n_cand = 0;
       __syncwarp();
 #pragma unroll
       for (int j = 0; j < NJ; ++j) {
-        const long long kh = __double_as_longlong(p[j]) >> kSplit;
+        const long long kh = __double_as_longlong(p[j]) >> low;
         if (kh > hi) {
           if (j & 1) ab1 += p[j]; else ab0 += p[j];
         }
         const bool is_c = (kh == hi) && (j * 32 + lane < nb);
         const unsigned bal = __ballot_sync(0xffffffffu, is_c);
-        if (is_c) scr[n_cand + __popc(bal & lt_mask)] = p[j];
+        if (is_c) {
+          const int pos = n_cand + __popc(bal & lt_mask);
+          if (pos < kMaxCand) scr[pos] = p[j];
+        }
         n_cand += __popc(bal);
       }
       const double mass_above = warp_sum(ab0 + ab1);
       __syncwarp();
-      if (n_cand <= 64) {
+      if (n_cand <= kMaxCand) {
         // Few candidates: each lane takes two of them and adds up, over all candidates, the mass at
         // or above its own value; theta is the largest candidate whose mass still reaches tau (the
         // smallest candidate always does: that is what the prefix search established).
@@ -262,10 +259,18 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
           best = other > best ? other : best;
         }
         theta = best;
-      } else {  // many near-equal blocks: keep searching over all of them
-        for (int bit = kSplit - 1; bit >= 0; --bit) {
-          const long long cand = theta | (1LL << bit);
-          if (mass_at_least(cand) >= t) theta = cand;
+      } else {  // many near-equal blocks: keep searching over all of them, a bit at a time
+        for (int bit = low - 1; bit >= 0; --bit) {
+          const long long cnd = theta | (1LL << bit);
+          double g0 = 0.0, g1 = 0.0, g2 = 0.0, g3 = 0.0;  // fixed 4-way split: same order on every run
+#pragma unroll
+          for (int j = 0; j < NJ; j += 4) {
+            if (__double_as_longlong(p[j]) >= cnd) g0 += p[j];
+            if (j + 1 < NJ && __double_as_longlong(p[j + 1]) >= cnd) g1 += p[j + 1];
+            if (j + 2 < NJ && __double_as_longlong(p[j + 2]) >= cnd) g2 += p[j + 2];
+            if (j + 3 < NJ && __double_as_longlong(p[j + 3]) >= cnd) g3 += p[j + 3];
+          }
+          if (warp_sum((g0 + g1) + (g2 + g3)) >= t) theta = cnd;
         }
       }
       double above = 0.0;
@@ -285,19 +290,27 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
         c += th;
         ++m_ties;
       } while (c < t && m_ties < nties);
+      n_ties = nties;
     }
 
     int base = 0, tie_seen = 0;
+    // the usual case: every block equal to theta is kept (theta = 0 when all blocks are kept)
+    const bool all_ties_kept = keep_all || m_ties == n_ties;
 #pragma unroll
     for (int j = 0; j < NJ; ++j) {
       const int J = j * 32 + lane;
       const long long b = __double_as_longlong(p[j]);
       const bool valid = J < nb;
-      const bool is_tie = valid && !keep_all && b == theta;
-      const unsigned tie_ballot = __ballot_sync(0xffffffffu, is_tie);
-      const int tie_rank = tie_seen + __popc(tie_ballot & lt_mask);
-      tie_seen += __popc(tie_ballot);
-      const bool keep = valid && (keep_all || b > theta || (is_tie && tie_rank < m_ties));
+      bool keep;
+      if (all_ties_kept) {
+        keep = valid && b >= theta;
+      } else {
+        const bool is_tie = valid && b == theta;
+        const unsigned tie_ballot = __ballot_sync(0xffffffffu, is_tie);
+        const int tie_rank = tie_seen + __popc(tie_ballot & lt_mask);
+        tie_seen += __popc(tie_ballot);
+        keep = valid && (b > theta || (is_tie && tie_rank < m_ties));
+      }
       const unsigned word = __ballot_sync(0xffffffffu, keep);
       if (lane == 0 && j < W) mask_bits[row * W + j] = word;
       if (keep) kv_idx[row * idx_stride + base + __popc(word & lt_mask)] = J;
@@ -309,26 +322,28 @@ __global__ void __launch_bounds__(256) predict_mask_kernel(const double *__restr
 
 template <int NJ>
 static cudaError_t launch_nj(const Geom &g, const Workspace &w, const double *tau, const uint8_t *refresh,
-                             heart_state st, cudaStream_t s) {
-  const size_t smem = sizeof(double) * ((size_t)TI * NJ * 32 + TI * kD + TJ * KLD);
-  cudaError_t e = cudaFuncSetAttribute(predict_mask_kernel<NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)smem);
-  if (e != cudaSuccess) return e;
-  dim3 grid((g.nb + TI - 1) / TI, g.R);
-  predict_mask_kernel<NJ><<<grid, 256, smem, s>>>(w.bsum, g.R, g.N, g.block, g.nb, g.scale, tau, refresh,
-                                                 g.flags, st.mask_bits, st.kv_idx, st.kv_cnt,
-                                                 g.idx_stride, g.W);
+                             heart_state st, int pitch, cudaStream_t s) {
+  dim3 grid((g.nb + kRowsPerCta - 1) / kRowsPerCta, g.R);
+  top_p_kernel<NJ><<<grid, 32 * kRowsPerCta, 0, s>>>(w.scores, g.nb, pitch, tau, refresh, g.flags, st.mask_bits,
+                                                     st.kv_idx, st.kv_cnt, g.idx_stride, g.W);
   return cudaGetLastError();
 }
 
 cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
                                 const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches) {
-  ++*launches;
-  const int nj = (g.nb + 31) / 32;
-  if (nj <= 8) return launch_nj<8>(g, w, tau, refresh, st, s);
-  if (nj <= 16) return launch_nj<16>(g, w, tau, refresh, st, s);
-  if (nj <= 24) return launch_nj<24>(g, w, tau, refresh, st, s);
-  return launch_nj<32>(g, w, tau, refresh, st, s);
+  *launches += 2;
+  const int nj = (g.nb + 31) / 32, pitch = nj * 32;
+  const size_t smem = sizeof(double) * 2 * (SI + SJ) * KLD;
+  cudaError_t e = cudaFuncSetAttribute(pooled_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid((g.nb + SJ - 1) / SJ, (g.nb + SI - 1) / SI, g.R);
+  pooled_scores_kernel<<<grid, 256, smem, s>>>(w.bmean, g.R, g.nb, pitch, g.scale, refresh, w.scores);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (nj <= 8) return launch_nj<8>(g, w, tau, refresh, st, pitch, s);
+  if (nj <= 16) return launch_nj<16>(g, w, tau, refresh, st, pitch, s);
+  if (nj <= 24) return launch_nj<24>(g, w, tau, refresh, st, pitch, s);
+  return launch_nj<32>(g, w, tau, refresh, st, pitch, s);
 }
 
 }  // namespace heart

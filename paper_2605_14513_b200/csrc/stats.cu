@@ -1,4 +1,4 @@
-// Streaming statistics of one layer-step: per-block sums of Q and K in a single pass over HBM
+// Streaming statistics of one layer-step: per-block means of Q and K in a single pass over HBM
 // (token-mean pooling of Algorithm 1 line 1 and the block pooling of the mask predictor share the
 // pass), then the mean-pooled L1 drift, the refresh-or-reuse decision, the layer gate and the
 // anchor update (Eq. mean-pooled drift; Algorithm 1; layer-level gating of the TMR section).
@@ -31,7 +31,7 @@ template <int BLOCK>
 __global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restrict__ Q,
                                                          const uint16_t *__restrict__ K, long long sb,
                                                          long long sh, long long sn, int H, int N,
-                                                         int nb, int bpc, double *__restrict__ bsum,
+                                                         int nb, int bpc, double *__restrict__ bmean,
                                                          double *__restrict__ psum) {
   constexpr int ITERS = BLOCK / 16;
   const int chunk = blockIdx.x, r = blockIdx.y, z = blockIdx.z, R = gridDim.y;
@@ -55,7 +55,10 @@ __global__ void __launch_bounds__(256) block_sums_kernel(const uint16_t *__restr
     double s = 0.0;
 #pragma unroll
     for (int k = 0; k < 16; ++k) s += (double)sm[buf][k][threadIdx.x];
-    bsum[(((size_t)z * R + r) * nb + I) * kD + threadIdx.x] = s;
+    // the pooled mean of the block (what the mask predictor contracts); a full block divides by a
+    // power of two, exactly
+    const int rows = min(BLOCK, N - I * BLOCK);
+    bmean[(((size_t)z * R + r) * nb + I) * kD + threadIdx.x] = (rows == BLOCK) ? s * (1.0 / BLOCK) : s / (double)rows;
     total += s;
   };
   load_block(i0, cur);
@@ -196,9 +199,9 @@ cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, const
   dim3 grid(g.nchunks, g.R, 2);
   const uint16_t *q = static_cast<const uint16_t *>(Q), *k = static_cast<const uint16_t *>(K);
   if (g.block == 64)
-    block_sums_kernel<64><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bsum, w.psum);
+    block_sums_kernel<64><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bmean, w.psum);
   else
-    block_sums_kernel<128><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bsum, w.psum);
+    block_sums_kernel<128><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bmean, w.psum);
   ++*launches;
   return cudaGetLastError();
 }

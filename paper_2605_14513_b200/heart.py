@@ -24,7 +24,7 @@ SYMBOLS = (
     "heart_workspace_bytes", "heart_state_reset", "heart_drift", "heart_predict_mask",
     "heart_block_sparse_attn", "heart_step", "heart_step_host", "heart_get_status", "heart_strerror",
     "heart_last_launch_count", "heart_drift_static", "heart_full_token_drift", "heart_mask_iou",
-    "heart_band_error_workspace_bytes", "heart_band_error",
+    "heart_band_error_workspace_bytes", "heart_band_error", "heart_drift_workspace_bytes",
 )
 
 
@@ -60,6 +60,8 @@ def lib():
         l = C.CDLL(_LIB_PATH)
         l.heart_workspace_bytes.restype = C.c_size_t
         l.heart_workspace_bytes.argtypes = [C.POINTER(Config)]
+        l.heart_drift_workspace_bytes.restype = C.c_size_t
+        l.heart_drift_workspace_bytes.argtypes = [C.POINTER(Config)]
         l.heart_strerror.restype = C.c_char_p
         l.heart_strerror.argtypes = [C.c_int]
         l.heart_last_launch_count.restype = C.c_int
@@ -146,6 +148,11 @@ class State:
 
 def workspace_bytes(cfg: Config) -> int:
     return int(lib().heart_workspace_bytes(C.byref(cfg)))
+
+
+def drift_workspace_bytes(cfg: Config) -> int:
+    """The leading part of the workspace that heart_drift alone touches."""
+    return int(lib().heart_drift_workspace_bytes(C.byref(cfg)))
 
 
 def new_workspace(cfg: Config, device="cuda") -> torch.Tensor:
