@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
   if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: mask untouched
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   __shared__ double cand[kRowsPerCta][kMaxCand];
+  __shared__ uint16_t kept[kRowsPerCta][NJ * 32];
   const unsigned lt_mask = (1u << lane) - 1u;
   {
     const int I = blockIdx.x * kRowsPerCta + warp;
@@ -296,6 +297,11 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
     int base = 0, tie_seen = 0;
     // the usual case: every block equal to theta is kept (theta = 0 when all blocks are kept)
     const bool all_ties_kept = keep_all || m_ties == n_ties;
+    // The kept indices are gathered in shared memory and the mask words in registers (lane l keeps
+    // word l), so that the row leaves in a few coalesced stores.
+    uint16_t *lst = kept[warp];
+    uint32_t my_word = 0u;
+    __syncwarp();
 #pragma unroll
     for (int j = 0; j < NJ; ++j) {
       const int J = j * 32 + lane;
@@ -312,10 +318,13 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
         keep = valid && (b > theta || (is_tie && tie_rank < m_ties));
       }
       const unsigned word = __ballot_sync(0xffffffffu, keep);
-      if (lane == 0 && j < W) mask_bits[row * W + j] = word;
-      if (keep) kv_idx[row * idx_stride + base + __popc(word & lt_mask)] = J;
+      if (lane == j) my_word = word;
+      if (keep) lst[base + __popc(word & lt_mask)] = (uint16_t)J;
       base += __popc(word);
     }
+    __syncwarp();
+    if (lane < W) mask_bits[row * W + lane] = my_word;
+    for (int k = lane; k < base; k += 32) kv_idx[row * idx_stride + k] = lst[k];
     if (lane == 0) kv_cnt[row] = base;
   }
 }
