@@ -219,6 +219,23 @@ def test_uniform_scores_keep_lowest_indices(heart, oracle):
     assert np.all(mask_bits_u32(p.gst.mask_bits)[:, :, 0] == (1 << 29) - 1)
 
 
+def test_many_tied_blocks_around_the_threshold(heart, oracle):
+    """100 key blocks of which 90 have identical keys (identical pooled means, so identical weights
+    down to the last bit): the threshold falls inside the tie group for the larger tau, more candidates
+    share its leading bits than the direct evaluation takes, and ties must enter lowest index first."""
+    wl = inputs.small_workload(H=3, grid=(5, 16, 80), block=64, seed=21, tau=[0.3, 0.9, 0.995], pos_scale=0.5)
+    assert wl.n_blocks == 100
+    p = Pair(wl, heart, oracle)
+    K = p.K.clone()
+    K[:, :, 640:, :] = K[:, :, 640:704, :].repeat(1, 1, 90, 1)
+    p.K, p.Kb = K, inputs.bits(K)
+    p.gpu_step(want_lse=False)
+    p.oracle_step(want_O=False)
+    assert check_masks(p.gst, p.ost, range(wl.R), wl.tau, p.probs_row) == 0
+    cnt = to_np(p.gst.kv_cnt)
+    assert cnt.min() >= 1 and cnt.max() > 64  # some rows cut inside the tie group, beyond 64 candidates
+
+
 def test_layer_gate_on_gpu(heart, oracle):
     wl = inputs.small_workload(H=5, grid=(2, 9, 13), block=64, seed=9, eps=[0.3, 0.001, 0.001, 0.001, 0.001],
                                delta=np.full(5, 1.0))
