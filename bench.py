@@ -209,11 +209,14 @@ def run_ours(args, rank, world):
     ms_per_step = total_ms / K
 
     # ---- per-stage pass: the same K steps as three C-ABI calls, one event pair per call.  Nothing here
-    # synchronises with the host: the flop / pair / refresh counts are accumulated on the device.
+    # synchronises with the host, and nothing but the three calls and the event records is enqueued (the
+    # accounting kernels of the pass after it would otherwise sit between a step's attention and the next
+    # step's drift call and stretch the latter's interval by ~14 us).
     st.load_state_dict(ckpt)
     stage_ev = []
-    acc = torch.zeros(3, dtype=torch.float64, device=dev)  # retained flops, retained pairs, refreshed heads
     r2 = torch.empty_like(refresh)
+    torch.cuda.synchronize()
+    sampler2 = ClockSampler(uuid) if rank == 0 else None  # this pass has its own clock record
     for k in range(K):
         Q, Kt, V = steps_in[W + k]
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
@@ -225,6 +228,16 @@ def run_ours(args, rank, world):
         heart.heart_block_sparse_attn(cfg, Q, Kt, V, st.kv_idx, st.kv_cnt, O, ws)
         e[3].record()
         stage_ev.append(e)
+    torch.cuda.synchronize()
+    clocks_stage = sampler2.stop() if sampler2 else None
+    # ---- accounting pass (untimed): the same decisions and masks again from the same state; the flop /
+    # pair / refresh counts are accumulated on the device.
+    st.load_state_dict(ckpt)
+    acc = torch.zeros(3, dtype=torch.float64, device=dev)  # retained flops, retained pairs, refreshed heads
+    for k in range(K):
+        Q, Kt, V = steps_in[W + k]
+        heart.heart_drift(cfg, Q, Kt, delta, st, ws, refresh_out=r2)
+        heart.heart_predict_mask(cfg, Q, Kt, tau, st, ws, refresh=r2)
         f, p = retained_flops(torch, st, wl)
         acc += torch.stack([f, p, r2.sum().to(torch.float64)])
     torch.cuda.synchronize()
@@ -312,7 +325,8 @@ def run_ours(args, rank, world):
                                "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm / pk["hbm_gbs"],
                                "frac_of_nominal_8TBps": hbm / 8000.0, "bytes_per_launch": stats_bytes,
                                "ms_per_launch": ms_drift},
-            "gpu_launches": launches, "wall_ms_timed_region": wall_ms, "clocks": clocks, "e2e": e2e,
+            "gpu_launches": launches, "wall_ms_timed_region": wall_ms, "clocks": clocks,
+            "clocks_stage_pass": clocks_stage, "e2e": e2e,
         }
     return out, (wl, steps_in, W)
 
