@@ -84,6 +84,8 @@ struct AttnParams {
   long long sb, sh, sn;
   int H, N, nb, idx_stride, n_ctas_per_head, dense;
   int h0, hcount, R_all;  // this launch covers heads [h0, h0 + hcount) of every batch entry; R_all = B*H
+  const int32_t *order;   // the last n_sorted CTAs take their tile from this table (longest lists first)
+  int n_sorted;
   float scale_log2;
 };
 
@@ -127,7 +129,15 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
   // same role (above all the issuer of the score products) on the same sub-partition.
   const int kWarpKProd = 4 + ((kRoleKProd + blockIdx.x) & 3), kWarpVProd = 4 + ((kRoleVProd + blockIdx.x) & 3),
             kWarpPV = 4 + ((kRolePV + blockIdx.x) & 3), kWarpQK = 4 + ((kRoleQK + blockIdx.x) & 3);
-  const int rr = blockIdx.x / p.n_ctas_per_head, cta_in_head = blockIdx.x % p.n_ctas_per_head;
+  // Tiles run head-major, which keeps the K/V of one or two heads in L2.  Only the tiles of the
+  // last two heads are taken longest-first from a table: the launch then ends on short tiles
+  // instead of waiting for a long one that started late.
+  int tile = blockIdx.x;
+  {
+    const int first_sorted = (int)gridDim.x - p.n_sorted;
+    if (tile >= first_sorted) tile = first_sorted + __ldg(&p.order[tile - first_sorted]);
+  }
+  const int rr = tile / p.n_ctas_per_head, cta_in_head = tile % p.n_ctas_per_head;
   const int bidx = rr / p.hcount, hidx = p.h0 + rr % p.hcount;
   const int r = bidx * p.H + hidx;
   const int row0 = cta_in_head * 128;  // first query token of this CTA
@@ -556,6 +566,31 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
   if (tid == 0 && bars->abort) atomicExch(p.status, HEART_ERR_DEVICE_CHECK);
 }
 
+// Order of the last `n` tiles of a launch (those of its last one or two heads): descending by the
+// number of listed key blocks, ties by tile index -- rank by counting, so `order` is a permutation
+// whatever the counts hold.  n <= 2048.
+__global__ void __launch_bounds__(256) tail_order_kernel(const int32_t *__restrict__ kv_cnt, int nb, int qbt, int ncph,
+                                                         int idx_stride, int H, int h0, int hcount, int rr0, int n,
+                                                         int32_t *__restrict__ order) {
+  __shared__ int key[2048];
+  for (int t = threadIdx.x; t < n; t += blockDim.x) {
+    const int rr = rr0 + t / ncph, r = (rr / hcount) * H + h0 + rr % hcount;
+    int k = 0;
+    for (int qb = 0; qb < qbt; ++qb) {
+      const int I = (t % ncph) * qbt + qb;
+      if (I < nb) k += min(max(kv_cnt[(size_t)r * nb + I], 0), idx_stride);
+    }
+    key[t] = k;
+  }
+  __syncthreads();
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= n) return;
+  const int mine = key[t];
+  int rank = 0;
+  for (int u = 0; u < n; ++u) rank += (key[u] > mine || (key[u] == mine && u < t)) ? 1 : 0;
+  order[rank] = t;
+}
+
 // ---------------------------------------------------------------------- host side
 namespace {
 
@@ -606,7 +641,8 @@ cudaError_t launch_bk(const Geom &g, const CUtensorMap &mq, const CUtensorMap &m
 
 cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const void *V,
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,
-                             float *lse, int32_t *status, cudaStream_t s, int *launches, int h0, int hcount) {
+                             float *lse, int32_t *status, int32_t *order, cudaStream_t s, int *launches, int h0,
+                             int hcount) {
   if (hcount <= 0) {
     h0 = 0;
     hcount = g.H;
@@ -633,6 +669,19 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
   prm.hcount = hcount;
   prm.R_all = g.R;
   prm.scale_log2 = (float)(g.scale * 1.4426950408889634);
+  prm.order = order;
+  prm.n_sorted = 0;
+  if (!dense && order != nullptr) {
+    const int rows = g.B * hcount, nlast = rows < 2 ? rows : 2, n = nlast * prm.n_ctas_per_head;
+    if (n <= 2048) {
+      tail_order_kernel<<<(n + 255) / 256, 256, 0, s>>>(kv_cnt, g.nb, 128 / g.block, prm.n_ctas_per_head, g.idx_stride,
+                                                        g.H, h0, hcount, rows - nlast, n, order);
+      cudaError_t e = cudaGetLastError();
+      if (e != cudaSuccess) return e;
+      prm.n_sorted = n;
+      ++*launches;
+    }
+  }
   ++*launches;
   return g.block == 64 ? launch_bk<64>(g, mq, mk, mv, prm, s) : launch_bk<128>(g, mq, mk, mv, prm, s);
 }

@@ -43,6 +43,7 @@ struct Workspace {
   uint8_t *pre;       // [R]            head-wise decision before the gate
   uint8_t *refresh;   // [R]            final decision of the current step
   double *drift;      // [R]
+  int32_t *order;     // [2048] tile order of the last two heads of an attention launch
   double *scores;     // [R][nb][pitch] pooled scores of the refreshed heads, pitch = nb rounded up to 32
   size_t bytes_drift;  // what heart_drift alone touches (everything above `scores`)
   size_t bytes;
@@ -70,6 +71,8 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   off += align256((size_t)g.R);
   w.drift = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * (size_t)g.R);
+  w.order = reinterpret_cast<int32_t *>(p + off);
+  off += align256(sizeof(int32_t) * 2048);
   w.bytes_drift = off;
   w.scores = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * (size_t)g.R * g.nb * (size_t)(((g.nb + 31) / 32) * 32));
@@ -88,8 +91,8 @@ cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double 
 // h0/hcount select the heads [h0, h0 + hcount) of every batch entry (hcount <= 0: all heads).
 cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const void *V,
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,
-                             float *lse, int32_t *status, cudaStream_t s, int *launches, int h0 = 0,
-                             int hcount = 0);
+                             float *lse, int32_t *status, int32_t *order, cudaStream_t s, int *launches,
+                             int h0 = 0, int hcount = 0);
 
 cudaError_t launch_token_drift(const Geom &g, const void *Qa, const void *Ka, const void *Qb,
                                const void *Kb, double *partial, double *drift_out, cudaStream_t s,

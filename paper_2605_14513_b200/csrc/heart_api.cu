@@ -150,7 +150,7 @@ int heart_block_sparse_attn(const heart_config *cfg, const void *Q, const void *
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   Workspace w = carve(g, workspace);
   g_launches = 0;
-  cudaError_t e = launch_attention(g, Q, K, V, kv_idx, kv_cnt, dense, O, lse, w.status, s, &g_launches);
+  cudaError_t e = launch_attention(g, Q, K, V, kv_idx, kv_cnt, dense, O, lse, w.status, w.order, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "attention");
   return HEART_OK;
 }
@@ -173,7 +173,7 @@ int heart_step(const heart_config *cfg, const void *Q, const void *K, const void
     fill_dense_outputs_kernel<<<(g.R + 127) / 128, 128, 0, s>>>(g.R, drift_out, refresh_out, w.refresh);
     ++g_launches;
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "fill_dense_outputs");
-    e = launch_attention(g, Q, K, V, nullptr, nullptr, true, O, lse, w.status, s, &g_launches);
+    e = launch_attention(g, Q, K, V, nullptr, nullptr, true, O, lse, w.status, w.order, s, &g_launches);
     if (e != cudaSuccess) return cuda_fail(e, "attention");
     return HEART_OK;
   }
@@ -183,7 +183,7 @@ int heart_step(const heart_config *cfg, const void *Q, const void *K, const void
   if (e != cudaSuccess) return cuda_fail(e, "decide");
   e = launch_predict_mask(g, w, tau, w.refresh, *st, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
-  e = launch_attention(g, Q, K, V, st->kv_idx, st->kv_cnt, false, O, lse, w.status, s, &g_launches);
+  e = launch_attention(g, Q, K, V, st->kv_idx, st->kv_cnt, false, O, lse, w.status, w.order, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "attention");
   return HEART_OK;
 }
@@ -281,7 +281,7 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
     if (e == cudaSuccess) e = cudaStreamWaitEvent(s, pp->ev_v[gi], 0);
     if (e != cudaSuccess) return cuda_fail(e, "heart_step_host (host to device)");
     e = launch_attention(g, Q_dev, K_dev, V_dev, dense ? nullptr : st->kv_idx, dense ? nullptr : st->kv_cnt, dense,
-                         O_dev, nullptr, w.status, s, &g_launches, h0, h1 - h0);
+                         O_dev, nullptr, w.status, w.order, s, &g_launches, h0, h1 - h0);
     if (e != cudaSuccess) return cuda_fail(e, "attention");
     e = cudaEventRecord(pp->ev_o[gi], s);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(pp->s_out, pp->ev_o[gi], 0);
