@@ -568,27 +568,29 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
 
 // Order of the last `n` tiles of a launch (those of its last one or two heads): descending by the
 // number of listed key blocks, ties by tile index -- rank by counting, so `order` is a permutation
-// whatever the counts hold.  n <= 2048.
+// whatever the counts hold.  n <= 2048.  Eight threads share a tile (each counts an eighth of the
+// keys), 32 tiles per CTA.
 __global__ void __launch_bounds__(256) tail_order_kernel(const int32_t *__restrict__ kv_cnt, int nb, int qbt, int ncph,
                                                          int idx_stride, int H, int h0, int hcount, int rr0, int n,
                                                          int32_t *__restrict__ order) {
   __shared__ int key[2048];
   for (int t = threadIdx.x; t < n; t += blockDim.x) {
     const int rr = rr0 + t / ncph, r = (rr / hcount) * H + h0 + rr % hcount;
+    const int I0 = (t % ncph) * qbt;
     int k = 0;
-    for (int qb = 0; qb < qbt; ++qb) {
-      const int I = (t % ncph) * qbt + qb;
-      if (I < nb) k += min(max(kv_cnt[(size_t)r * nb + I], 0), idx_stride);
-    }
+    if (I0 < nb) k += min(max(__ldg(&kv_cnt[(size_t)r * nb + I0]), 0), idx_stride);
+    if (qbt == 2 && I0 + 1 < nb) k += min(max(__ldg(&kv_cnt[(size_t)r * nb + I0 + 1]), 0), idx_stride);
     key[t] = k;
   }
   __syncthreads();
-  const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= n) return;
-  const int mine = key[t];
+  const int t = blockIdx.x * 32 + (threadIdx.x >> 3), part = threadIdx.x & 7;
+  const int mine = t < n ? key[t] : 0;
   int rank = 0;
-  for (int u = 0; u < n; ++u) rank += (key[u] > mine || (key[u] == mine && u < t)) ? 1 : 0;
-  order[rank] = t;
+  for (int u = part; u < n; u += 8) rank += (key[u] > mine || (key[u] == mine && u < t)) ? 1 : 0;
+  rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+  rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+  rank += __shfl_xor_sync(0xffffffffu, rank, 4);
+  if (part == 0 && t < n) order[rank] = t;
 }
 
 // ---------------------------------------------------------------------- host side
@@ -674,7 +676,7 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
   if (!dense && order != nullptr) {
     const int rows = g.B * hcount, nlast = rows < 2 ? rows : 2, n = nlast * prm.n_ctas_per_head;
     if (n <= 2048) {
-      tail_order_kernel<<<(n + 255) / 256, 256, 0, s>>>(kv_cnt, g.nb, 128 / g.block, prm.n_ctas_per_head, g.idx_stride,
+      tail_order_kernel<<<(n + 31) / 32, 256, 0, s>>>(kv_cnt, g.nb, 128 / g.block, prm.n_ctas_per_head, g.idx_stride,
                                                         g.H, h0, hcount, rows - nlast, n, order);
       cudaError_t e = cudaGetLastError();
       if (e != cudaSuccess) return e;
