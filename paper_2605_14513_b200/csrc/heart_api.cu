@@ -191,7 +191,7 @@ int heart_step(const heart_config *cfg, const void *Q, const void *K, const void
 namespace {
 
 // Streams and events of heart_step_host, created on first use on each device and kept.
-constexpr int kHostGroups = 4;  // head groups the V copy, the attention and the O copy are pipelined over
+constexpr int kHostGroups = 16;  // head groups the V copy, the attention and the O copy are pipelined over
 struct HostPipe {
   bool ready = false;
   cudaStream_t s_in = nullptr, s_out = nullptr;
