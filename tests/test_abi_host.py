@@ -45,6 +45,13 @@ def test_workspace_size_and_shape_validation(heart):
     assert heart.workspace_bytes(heart.make_config(1, 1, 64 * 1025, 64)) == 0         # too many blocks
     assert heart.workspace_bytes(heart.make_config(1, 1, 64 * 1024, 64)) > 0
     assert heart.workspace_bytes(heart.make_config(1, 0, 128, 64)) == 0
+    # the drift-only prefix: block means, token means, flags -- without the pooled scores of the mask
+    # predictor (8 bytes per (head, query block, key block) with the key blocks padded to 32)
+    d = heart.drift_workspace_bytes(cfg)
+    assert 2 * 12 * nb * 128 * 8 <= d < n and d % 256 == 0
+    assert n - d == 12 * nb * nb * 8
+    assert d <= 16 << 20                                                               # fits the built-in scratch
+    assert heart.drift_workspace_bytes(heart.make_config(1, 12, 32760, 32)) == 0
 
 
 def test_bad_arguments_are_rejected_on_the_host(heart):
