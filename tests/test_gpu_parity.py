@@ -89,6 +89,26 @@ def test_small_sweeps(heart, oracle, block, grid, H, B):
     assert ex_rows == 0 and ex_flags == 0
 
 
+def test_random_small_shapes(heart, oracle):
+    """24 seeded random shapes (both block sizes, ragged token counts, 1-3 heads, one or two batch
+    entries, gate on or off, padded index pitch), three steps each, everything compared in full."""
+    rs = np.random.RandomState(20260514)
+    for case in range(24):
+        block = int(rs.choice([64, 128]))
+        grid = (int(rs.randint(1, 7)), int(rs.randint(3, 30)), int(rs.randint(3, 44)))
+        N = grid[0] * grid[1] * grid[2]
+        H, B = int(rs.randint(1, 4)), int(rs.choice([1, 1, 2]))
+        R = B * H
+        wl = inputs.small_workload(H=H, grid=grid, block=block, seed=int(rs.randint(1, 10000)), steps=3, B=B,
+                                   eps=np.exp(rs.uniform(np.log(0.003), np.log(0.3), R)),
+                                   tau=rs.uniform(0.3, 0.995, R), delta=np.full(R, 0.8 * np.sqrt(420.0 / N)),
+                                   pos_scale=float(rs.choice([0.5, 1.5, 2.5, 3.0])))
+        pair = Pair(wl, heart, oracle, idx_pad=int(rs.randint(0, 7)),
+                    gate=(0.0, 1.0) if rs.rand() < 0.5 else (0.4, 0.8))
+        _, ex_rows, ex_flags = run_sweep(pair, 3)
+        assert ex_rows == 0 and ex_flags == 0, (case, block, grid, H, B)
+
+
 def test_tiny_config_in_full(heart, oracle):
     """Config 1: H=2, N=2048, block 64; step 0 both refresh, step 1 only head 1."""
     pair = Pair(inputs.workload("tiny"), heart, oracle)
