@@ -74,6 +74,7 @@ struct AttnBars {
   int n_union;
   int abort;
   int bad;
+  int first_j;  // key block whose K tile was requested before the step list existed (-1: none)
 };
 
 struct AttnParams {
@@ -190,6 +191,23 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
     tma_load_4d(Qs, &map_q, &bars->q_full, 0, row0, hidx, bidx);
     tma_load_4d(Qs + 128 * 128, &map_q, &bars->q_full, 64, row0, hidx, bidx);
   }
+  if (tid == 0) {
+    // Thread 0 holds the first entry of each list.  Whatever the union turns out to be, that key
+    // block is in it: its K tile is requested now, ~2000 clocks before the step list is ready, and
+    // the compaction below puts the block first (for ascending lists it is the first anyway).
+    int j0 = 0x7fffffff;
+#pragma unroll
+    for (int qb = 0; qb < L::QBT; ++qb)
+      if (cnt_q[qb] > 0 && p.idx_stride > 0) j0 = min(j0, ent[qb][0] < 0 ? 0x7fffffff : ent[qb][0]);
+    if (j0 < nb) {
+      mbar_expect_tx(&bars->k_full[0], L::KV_BYTES);
+      tma_load_4d(Ks, &map_kv, &bars->k_full[0], 0, j0 * B, hidx, bidx);
+      tma_load_4d(Ks + kStep * 128, &map_kv, &bars->k_full[0], 64, j0 * B, hidx, bidx);
+      bars->first_j = j0;
+    } else {
+      bars->first_j = -1;
+    }
+  }
 #pragma unroll
   for (int qb = 0; qb < L::QBT; ++qb) {  // scatter: flag bit qb of every key block listed by query block qb
     const int I = cta_in_head * L::QBT + qb;
@@ -245,11 +263,21 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
       const int v = __shfl_up_sync(0xffffffffu, incl, o);
       if (lane >= o) incl += v;
     }
+    // the block whose K tile is already on its way goes first: p0 = its ascending rank
+    const int first_j = bars->first_j;
+    int p0 = 0;
+    if (first_j >= 0) {
+      const unsigned in_chunk = __ballot_sync(0xffffffffu, tbl[(first_j & ~31) + lane] != 0u);
+      p0 = __shfl_sync(0xffffffffu, incl - mine, first_j >> 5) + __popc(in_chunk & ((1u << (first_j & 31)) - 1u));
+    }
 #pragma unroll
     for (int i = 0; i < kChunksPerWarp; ++i) {
       const int chunk = warp + i * (kAttnThreads / 32);
       const int base = __shfl_sync(0xffffffffu, incl - mine, chunk);
-      if (f[i] != 0u) uni[base + __popc(ballot[i] & ((1u << lane) - 1u))] = (chunk * 32 + lane) | (int)(f[i] << 16);
+      if (f[i] != 0u) {
+        const int J = chunk * 32 + lane, q = base + __popc(ballot[i] & ((1u << lane) - 1u));
+        uni[J == first_j ? 0 : (q < p0 ? q + 1 : q)] = J | (int)(f[i] << 16);
+      }
     }
     const int total = __shfl_sync(0xffffffffu, incl, 31);
     if (tid == 0) {
@@ -281,6 +309,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
       int issued = 0;
       for (int h = 0; h < NH; ++h) {
         const int s = h % kStages, ph = (h / kStages) & 1;
+        if (h == 0 && bars->first_j >= 0) {  // requested during set-up
+          issued = 1;
+          continue;
+        }
         // the stage is free once S_{h-4} = Q K_{h-4}^T is complete
         if (h >= kStages && !mbar_wait_relaxed(&bars->qk_done[s], ph ^ 1, abort)) break;
         const int key0 = key0_of(h);
