@@ -183,6 +183,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
   }
   for (int j = tid; j < nb; j += kAttnThreads) tbl[j] = 0u;
   __syncthreads();
+  if (tid == 0) HEART_TR(1, 28);
   if (warp == kWarpKProd && lane == 0) {  // the Q tile does not depend on the lists: start it now
     tma_prefetch_desc(&map_q);
     tma_prefetch_desc(&map_kv);
@@ -238,11 +239,13 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
       }
     }
   }
+  if (tid == 0) HEART_TR(1, 29);
   if (warp == kWarpQK) {
     tmem_alloc(&bars->tmem_base, kTmemCols);
     tmem_relinquish();
   }
   __syncthreads();
+  if (tid == 0) HEART_TR(1, 30);
   {  // ascending compaction of the flagged key blocks: warp w takes the 32-block chunks w, w+16
     constexpr int kChunksPerWarp = kMaxNb / 32 / (kAttnThreads / 32);
     uint32_t f[kChunksPerWarp];
