@@ -35,6 +35,35 @@ __device__ __forceinline__ double warp_max(double v) {
   return v;
 }
 
+// exp(x) for x <= 0 in about a third of the instructions of the library routine, which spends most of
+// its time on ranges that cannot occur here: n = rint(x log2 e) by the magic-number add, r = x - n ln 2
+// in two steps, the Taylor polynomial of degree 13 on |r| <= ln 2 / 2 (truncation 4e-18), 2^n by an
+// integer add into the exponent field.  Below -708 (weights under 1e-307 of the row maximum) it
+// returns 0.  Within an ulp or two of the correctly rounded value, like the library routine.
+__device__ __forceinline__ double exp_nonpositive(double x) {
+  if (x < -708.0) return 0.0;
+  const double t = fma(x, 1.4426950408889634, 6755399441055744.0);
+  const int n = __double2loint(t);
+  const double fn = t - 6755399441055744.0;
+  double r = fma(fn, -6.93147180369123816490e-01, x);
+  r = fma(fn, -1.90821492927058770002e-10, r);
+  double q = 1.6059043836821613e-10;            // 1/13!
+  q = fma(q, r, 2.08767569878681e-09);          // 1/12!
+  q = fma(q, r, 2.505210838544172e-08);         // 1/11!
+  q = fma(q, r, 2.755731922398589e-07);         // 1/10!
+  q = fma(q, r, 2.7557319223985893e-06);        // 1/9!
+  q = fma(q, r, 2.48015873015873e-05);          // 1/8!
+  q = fma(q, r, 1.984126984126984e-04);         // 1/7!
+  q = fma(q, r, 1.388888888888889e-03);         // 1/6!
+  q = fma(q, r, 8.333333333333333e-03);         // 1/5!
+  q = fma(q, r, 4.1666666666666664e-02);        // 1/4!
+  q = fma(q, r, 1.6666666666666666e-01);        // 1/3!
+  q = fma(q, r, 0.5);
+  q = fma(q, r, 1.0);
+  q = fma(q, r, 1.0);
+  return __hiloint2double(__double2hiint(q) + (n << 20), __double2loint(q));
+}
+
 // 8-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead
 __device__ __forceinline__ void cp_async8(double *smem_dst, const double *src, int src_bytes) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),
@@ -127,30 +156,34 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
   const int r = blockIdx.y;
   if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: mask untouched
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  extern __shared__ __align__(16) unsigned char smem_top[];
+  double *weights = reinterpret_cast<double *>(smem_top);  // [kRowsPerCta][NJ * 32]
   __shared__ double cand[kRowsPerCta][kMaxCand];
-  __shared__ uint16_t kept[kRowsPerCta][NJ * 32];
   const unsigned lt_mask = (1u << lane) - 1u;
   {
     const int I = blockIdx.x * kRowsPerCta + warp;
     if (I >= nb) return;
     const size_t row = (size_t)r * nb + I;
     const double *srow = scores + row * pitch;
-    double p[NJ];
+    // The weights of the row live in shared memory (lane-major, conflict-free): rolled loops over the
+    // NJ blocks of a lane keep the kernel small enough for the instruction cache -- fully unrolled
+    // over registers it was several times slower at n_b > 512.
+    double *pw = weights + (size_t)warp * NJ * 32 + lane;
     const double neg_inf = __longlong_as_double(0xfff0000000000000LL);
     double mx = neg_inf;
-#pragma unroll
+#pragma unroll 4
     for (int j = 0; j < NJ; ++j) {
       const int J = j * 32 + lane;
-      p[j] = (J < nb) ? srow[J] : neg_inf;
-      mx = fmax(mx, p[j]);
+      pw[(j) * 32] = (J < nb) ? srow[J] : neg_inf;
+      mx = fmax(mx, pw[(j) * 32]);
     }
     mx = warp_max(mx);
     double z = 0.0;
-#pragma unroll
+#pragma unroll 4
     for (int j = 0; j < NJ; ++j) {
       const int J = j * 32 + lane;
-      p[j] = (J < nb) ? exp(p[j] - mx) : 0.0;
-      z += p[j];
+      pw[(j) * 32] = (J < nb) ? exp_nonpositive(pw[(j) * 32] - mx) : 0.0;
+      z += pw[(j) * 32];
     }
     z = warp_sum(z);
     // From here on p holds the unnormalised weights e = exp(s - max) <= 1 and every mass is compared
@@ -170,15 +203,15 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
         const long long c1 = theta | (1LL << bit), c2 = theta | (2LL << bit), c3 = theta | (3LL << bit);
         const int h1 = (int)(c1 >> 32), h2 = (int)(c2 >> 32), h3 = (int)(c3 >> 32);
         double a1 = 0.0, a2 = 0.0, a3 = 0.0, b1 = 0.0, b2 = 0.0, b3 = 0.0;
-#pragma unroll
+#pragma unroll 2
         for (int j = 0; j < NJ; j += 2) {
-          const int k0 = __double2hiint(p[j]), k1 = __double2hiint(p[j + 1]);
-          if (k0 >= h1) a1 += p[j];
-          if (k0 >= h2) a2 += p[j];
-          if (k0 >= h3) a3 += p[j];
-          if (k1 >= h1) b1 += p[j + 1];
-          if (k1 >= h2) b2 += p[j + 1];
-          if (k1 >= h3) b3 += p[j + 1];
+          const int k0 = __double2hiint(pw[(j) * 32]), k1 = __double2hiint(pw[(j + 1) * 32]);
+          if (k0 >= h1) a1 += pw[(j) * 32];
+          if (k0 >= h2) a2 += pw[(j) * 32];
+          if (k0 >= h3) a3 += pw[(j) * 32];
+          if (k1 >= h1) b1 += pw[(j + 1) * 32];
+          if (k1 >= h2) b2 += pw[(j + 1) * 32];
+          if (k1 >= h3) b3 += pw[(j + 1) * 32];
         }
         double m1 = a1 + b1, m2 = a2 + b2, m3 = a3 + b3;
 #pragma unroll
@@ -198,9 +231,9 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
       int first_bit = 60;
       {
         int hmax = 0, hmin = 0x7fffffff;
-#pragma unroll
+#pragma unroll 4
         for (int j = 0; j < NJ; ++j) {
-          const int h = __double2hiint(p[j]);
+          const int h = __double2hiint(pw[(j) * 32]);
           hmax = max(hmax, h);
           if (j * 32 + lane < nb) hmin = min(hmin, h);
         }
@@ -220,17 +253,17 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
       double ab0 = 0.0, ab1 = 0.0;
       int n_cand = 0;
       __syncwarp();
-#pragma unroll
+#pragma unroll 4
       for (int j = 0; j < NJ; ++j) {
-        const long long kh = __double_as_longlong(p[j]) >> low;
+        const long long kh = __double_as_longlong(pw[(j) * 32]) >> low;
         if (kh > hi) {
-          if (j & 1) ab1 += p[j]; else ab0 += p[j];
+          if (j & 1) ab1 += pw[(j) * 32]; else ab0 += pw[(j) * 32];
         }
         const bool is_c = (kh == hi) && (j * 32 + lane < nb);
         const unsigned bal = __ballot_sync(0xffffffffu, is_c);
         if (is_c) {
           const int pos = n_cand + __popc(bal & lt_mask);
-          if (pos < kMaxCand) scr[pos] = p[j];
+          if (pos < kMaxCand) scr[pos] = pw[(j) * 32];
         }
         n_cand += __popc(bal);
       }
@@ -264,22 +297,22 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
         for (int bit = low - 1; bit >= 0; --bit) {
           const long long cnd = theta | (1LL << bit);
           double g0 = 0.0, g1 = 0.0, g2 = 0.0, g3 = 0.0;  // fixed 4-way split: same order on every run
-#pragma unroll
+#pragma unroll 1
           for (int j = 0; j < NJ; j += 4) {
-            if (__double_as_longlong(p[j]) >= cnd) g0 += p[j];
-            if (j + 1 < NJ && __double_as_longlong(p[j + 1]) >= cnd) g1 += p[j + 1];
-            if (j + 2 < NJ && __double_as_longlong(p[j + 2]) >= cnd) g2 += p[j + 2];
-            if (j + 3 < NJ && __double_as_longlong(p[j + 3]) >= cnd) g3 += p[j + 3];
+            if (__double_as_longlong(pw[(j) * 32]) >= cnd) g0 += pw[(j) * 32];
+            if (j + 1 < NJ && __double_as_longlong(pw[(j + 1) * 32]) >= cnd) g1 += pw[(j + 1) * 32];
+            if (j + 2 < NJ && __double_as_longlong(pw[(j + 2) * 32]) >= cnd) g2 += pw[(j + 2) * 32];
+            if (j + 3 < NJ && __double_as_longlong(pw[(j + 3) * 32]) >= cnd) g3 += pw[(j + 3) * 32];
           }
           if (warp_sum((g0 + g1) + (g2 + g3)) >= t) theta = cnd;
         }
       }
       double above = 0.0;
       int nties = 0;
-#pragma unroll
+#pragma unroll 4
       for (int j = 0; j < NJ; ++j) {
-        const long long b = __double_as_longlong(p[j]);
-        if (b > theta) above += p[j];
+        const long long b = __double_as_longlong(pw[(j) * 32]);
+        if (b > theta) above += pw[(j) * 32];
         nties += (b == theta && j * 32 + lane < nb) ? 1 : 0;
       }
       above = warp_sum(above);
@@ -297,15 +330,12 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
     int base = 0, tie_seen = 0;
     // the usual case: every block equal to theta is kept (theta = 0 when all blocks are kept)
     const bool all_ties_kept = keep_all || m_ties == n_ties;
-    // The kept indices are gathered in shared memory and the mask words in registers (lane l keeps
-    // word l), so that the row leaves in a few coalesced stores.
-    uint16_t *lst = kept[warp];
+    // The mask words are gathered in registers (lane l keeps word l) and leave in one store.
     uint32_t my_word = 0u;
-    __syncwarp();
-#pragma unroll
+#pragma unroll 4
     for (int j = 0; j < NJ; ++j) {
       const int J = j * 32 + lane;
-      const long long b = __double_as_longlong(p[j]);
+      const long long b = __double_as_longlong(pw[(j) * 32]);
       const bool valid = J < nb;
       bool keep;
       if (all_ties_kept) {
@@ -319,12 +349,10 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
       }
       const unsigned word = __ballot_sync(0xffffffffu, keep);
       if (lane == j) my_word = word;
-      if (keep) lst[base + __popc(word & lt_mask)] = (uint16_t)J;
+      if (keep) kv_idx[row * idx_stride + base + __popc(word & lt_mask)] = J;
       base += __popc(word);
     }
-    __syncwarp();
     if (lane < W) mask_bits[row * W + lane] = my_word;
-    for (int k = lane; k < base; k += 32) kv_idx[row * idx_stride + k] = lst[k];
     if (lane == 0) kv_cnt[row] = base;
   }
 }
@@ -333,7 +361,10 @@ template <int NJ>
 static cudaError_t launch_nj(const Geom &g, const Workspace &w, const double *tau, const uint8_t *refresh,
                              heart_state st, int pitch, cudaStream_t s) {
   dim3 grid((g.nb + kRowsPerCta - 1) / kRowsPerCta, g.R);
-  top_p_kernel<NJ><<<grid, 32 * kRowsPerCta, 0, s>>>(w.scores, g.nb, pitch, tau, refresh, g.flags, st.mask_bits,
+  const size_t smem = sizeof(double) * kRowsPerCta * NJ * 32;
+  cudaError_t e = cudaFuncSetAttribute(top_p_kernel<NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  top_p_kernel<NJ><<<grid, 32 * kRowsPerCta, smem, s>>>(w.scores, g.nb, pitch, tau, refresh, g.flags, st.mask_bits,
                                                      st.kv_idx, st.kv_cnt, g.idx_stride, g.W);
   return cudaGetLastError();
 }
