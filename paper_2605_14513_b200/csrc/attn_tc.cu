@@ -28,6 +28,11 @@
 // Tensor memory (256 columns per CTA): O | S[2]  =  128 + 2 x 64; key step h uses S[h & 1] and
 // shared-memory stage h & 1; P_h aliases S[h & 1].
 //
+// CTAs run head-major (the K/V of one or two heads stay in L2); the tiles of the last two heads of a
+// launch are taken longest-list-first from a table that tail_order_kernel writes just before, so that
+// the launch does not end on a long tile that started late.  The K tile of the first listed key block
+// is requested during set-up, before the step list is complete, and that block is put first.
+//
 // Every wait is bounded; a wait that runs out raises a CTA-wide abort flag and the status word, the
 // roles drain, tensor memory is freed and the CTA exits.
 #include <cuda.h>

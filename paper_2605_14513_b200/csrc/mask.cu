@@ -6,13 +6,15 @@
 // owns 64 query blocks x 128 key blocks of one head (each thread 8 x 4), the means arrive 16 dims at
 // a time by cp.async into a double-buffered shared-memory tile, and every score accumulates over the
 // 128 dims in ascending order in one fma chain.  The scores go to the workspace (they stay in L2).
-// top_p_kernel gives each warp one row: two-pass softmax, then top-p WITHOUT a sort: the kept set is
-// {p > theta} plus the lowest-index ties at theta, where theta is the largest element value whose
-// ">= theta" mass still reaches tau -- found by a search over the IEEE-754 pattern of p (positive
-// doubles order like their bit patterns): the top 14 bits two at a time over all blocks, the rest
-// directly over the few blocks that share that prefix.  Everything is fp64 so the integer outputs
-// (bit mask, ascending index list, count) agree with a plain fp64 sort-and-accumulate reference
-// except when the cumulative mass is within rounding (1e-15) of tau.
+// top_p_kernel gives each warp one row (its weights in shared memory, the loops over them rolled):
+// row max, unnormalised weights e = exp(s - max), then top-p WITHOUT a sort and without dividing by
+// the row sum z: the kept set is {e > theta} plus the lowest-index ties at theta, where theta is the
+// largest element value whose ">= theta" mass still reaches tau * z -- found by a search over the
+// IEEE-754 pattern of e (positive doubles order like their bit patterns): starting below the leading
+// bits that the largest and the smallest weight share, two bits a round over all blocks down to bit
+// 48, the rest directly over the few blocks that share that prefix.  Everything is fp64 so the
+// integer outputs (bit mask, ascending index list, count) agree with a plain fp64
+// sort-and-accumulate reference except when the cumulative mass is within rounding (1e-15) of tau.
 #include "common.cuh"
 
 namespace heart {
