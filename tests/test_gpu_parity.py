@@ -145,7 +145,7 @@ def test_step_equals_three_calls_and_checkpoint(heart, oracle):
         b.advance()
 
 
-@pytest.mark.parametrize("B,H,flags", [(1, 3, 0), (2, 5, 0), (1, 2, 2)])
+@pytest.mark.parametrize("B,H,flags", [(1, 3, 0), (2, 5, 0), (1, 2, 2), (1, 19, 0)])  # 19 heads: 16 uneven head groups
 def test_host_buffer_step_equals_device_step(heart, oracle, B, H, flags):
     """heart_step_host (uploads, per-head-group pipeline, downloads) against heart_step on the same
     bytes: identical O, drift, refresh and state at every step; the last row of flags runs the dense
