@@ -102,7 +102,7 @@ def test_random_small_shapes(heart, oracle):
         wl = inputs.small_workload(H=H, grid=grid, block=block, seed=int(rs.randint(1, 10000)), steps=3, B=B,
                                    eps=np.exp(rs.uniform(np.log(0.003), np.log(0.3), R)),
                                    tau=rs.uniform(0.3, 0.995, R), delta=np.full(R, 0.8 * np.sqrt(420.0 / N)),
-                                   pos_scale=float(rs.choice([0.5, 1.5, 2.5, 3.0])))
+                                   pos_scale=float(rs.choice([0.5, 1.5, 2.0, 2.5])))  # up to the workloads' value
         pair = Pair(wl, heart, oracle, idx_pad=int(rs.randint(0, 7)),
                     gate=(0.0, 1.0) if rs.rand() < 0.5 else (0.4, 0.8))
         _, ex_rows, ex_flags = run_sweep(pair, 3)
