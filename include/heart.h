@@ -16,8 +16,12 @@
  *
  * Conventions
  *   - Every pointer below is a DEVICE pointer owned by the caller unless it is
- *     marked "host".  The library never allocates or frees device memory and
- *     keeps no state between calls; all state lives in heart_state.
+ *     marked "host".  The library never allocates or frees device memory, and
+ *     everything the method carries from step to step lives in heart_state and
+ *     the caller's workspace.  What the library itself keeps, per device and
+ *     until the process exits: the two internal streams and the events of
+ *     heart_step_host (created by its first call), and the built-in scratch
+ *     array of heart_drift_static with its cached device address.
  *   - Every call except heart_get_status is asynchronous on `stream` and never
  *     synchronises.  Arguments are validated on the host before any launch;
  *     on a host-detected error nothing is launched and no state changes.
@@ -55,6 +59,10 @@ enum {
 #define HEART_FORCE_REFRESH 1u /* every head refreshes this step (decision overridden)  */
 #define HEART_FORCE_DENSE 2u   /* dense warm-up step (the baselines' first denoising    */
                                /* steps): attention over all blocks, TMR state untouched */
+#define HEART_BLOCK_MEANS_VALID 4u /* heart_predict_mask only: the workspace already holds */
+                               /* the block means of these Q, K (see that call)          */
+#define HEART_ESTIMATOR_ANTIDIAG 8u /* mask prediction ranks blocks with the strided       */
+                               /* antidiagonal estimator instead of mean pooling         */
 
 #define HEART_MAX_BLOCKS 1024  /* largest supported n_b */
 
@@ -110,9 +118,17 @@ int heart_drift(const heart_config *cfg, const void *Q, const void *K, const dou
  *   Qp[r,I,:] = mean of the real tokens of block I (same for Kp), fp64;
  *   P[r,I,:]  = softmax_J( scale * <Qp[r,I], Kp[r,J]> );
  *   keep the first k* blocks in (P descending, J ascending) order, k* = min{k>=1: cum mass >= tau[r]};
- *   tau[r] >= 1 (or a mass that never reaches tau) keeps all n_b blocks; at least one is kept.
+ *   tau[r] >= 1 (or NaN, or a mass that never reaches tau) keeps all n_b blocks; at least one is
+ *   kept: tau[r] <= 0 keeps exactly the largest block (the lowest index among equals).
  * Writes mask_bits, kv_idx (ascending), kv_cnt of those heads; other heads are untouched.
- * tau [R] fp64. */
+ * tau [R] fp64.
+ * The call first repeats heart_drift's pass over Q and K for the block means.  A caller that has just
+ * run heart_drift (or heart_predict_mask) on the same Q and K pointers, the same cfg shape and the
+ * same workspace, with no heart_full_token_drift and no change of the tensors' contents in between,
+ * sets HEART_BLOCK_MEANS_VALID in cfg->flags: the pass is skipped and the means in the workspace are
+ * used.  The kernels compare a signature of (pointers, shape, strides) that the pass left in the
+ * workspace; on a mismatch nothing is predicted and heart_get_status reports
+ * HEART_ERR_DEVICE_CHECK.  The contents of the tensors are the caller's promise. */
 int heart_predict_mask(const heart_config *cfg, const void *Q, const void *K, const double *tau,
                        const uint8_t *refresh, heart_state *st, void *workspace,
                        heart_stream_t stream);
@@ -170,7 +186,7 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
  * from a fixed HEART_STATIC_SCRATCH_BYTES array compiled into the library.  The call makes no
  * cudaMalloc / cudaFree and calls no allocating routine.
  *
- * Same arguments, results and error codes as heart_drift, except:
+ * Same arguments, results and error codes as heart_drift (an invalid cfg gives heart_drift's code), except:
  *   - no `workspace`; st->mask_bits / kv_idx / kv_cnt may be NULL (they are not touched);
  *   - a shape whose heart_drift_workspace_bytes exceeds HEART_STATIC_SCRATCH_BYTES is rejected with
  *     HEART_ERR_TOO_LARGE before anything is launched;
@@ -179,10 +195,12 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
  * The array is part of the library image: every GPU that loads the library holds those 16 MiB
  * until the process exits.  The first call on each device looks the array's device address up
  * (with that device current) and caches it; make that first call outside any stream capture.
- * All calls on a device share the one array and it keeps the previous call's contents: every
- * value the kernels read from it is rewritten by the same call first, so nothing needs clearing,
- * but two calls that overlap on the GPU (different streams, no ordering between them) race on it
- * and give undefined results -- serialise them. */
+ * All calls on a device share the one array and it keeps the previous call's contents.  Every
+ * value the kernels read from it is rewritten by the same call first, except one counter that the
+ * kernels expect to find at zero (the layer gate's ticket); each call clears it on `stream` before
+ * its kernels run.  Two calls that overlap on the GPU (different streams, no ordering between
+ * them) race on the array and give undefined results for both -- serialise them; calls after the
+ * race are sound again, because of that clearing. */
 int heart_drift_static(const heart_config *cfg, const void *Q, const void *K, const double *delta,
                        heart_state *st, double *drift_out, uint8_t *refresh_out, heart_stream_t stream);
 

@@ -18,14 +18,15 @@ struct Geom {
   int bpc, nchunks;  // block-sum kernel: key/query blocks per CTA and CTAs per (head row, tensor)
 };
 
-// Chunking of the block-sum pass: about 8 CTAs per SM on a 148-SM part, whatever the device (the
-// split fixes the summation order, so it must depend on the shape only).
+// Chunking of the block-sum pass: at most one wave of 5 CTAs per SM (48 registers x 256 threads) on a 148-SM part, whatever the
+// device (the split fixes the summation order, so it must depend on the shape only).  Never a little
+// more than one wave: the few CTAs of a second wave would each run as long as the whole first one.
 #ifndef HEART_CHUNK_TARGET
-#define HEART_CHUNK_TARGET (148 * 8)
+#define HEART_CHUNK_TARGET (148 * 5)
 #endif
 __host__ inline void set_chunks(Geom &g) {
   const int target = HEART_CHUNK_TARGET;
-  int per_pair = (target + 2 * g.R - 1) / (2 * g.R);
+  int per_pair = target / (2 * g.R);
   if (per_pair < 1) per_pair = 1;
   g.bpc = (g.nb + per_pair - 1) / per_pair;
   if (g.bpc < 1) g.bpc = 1;
@@ -35,11 +36,11 @@ __host__ inline void set_chunks(Geom &g) {
 // Workspace layout (all offsets 256-byte aligned).
 struct Workspace {
   int32_t *status;    // [64]   word 0: sticky device-check code; word 1: detail; word 8: ticket counter
-                      //        of the drift kernel (zero between launches)
+                      //        of the drift kernel (zero between launches); words 10-11: signature of
+                      //        the (Q, K, shape) whose block means the workspace holds (0: none)
   double *bmean;      // [2][R][nb][D]  per-block (pooled) means of Q (0) and K (1)
   double *psum;       // [2][R][nchunks][D]  per-CTA partial token sums
   double *mean;       // [2][R][D]      token means of the current step
-  double *part;       // [2][R]         L1 parts of the drift
   uint8_t *pre;       // [R]            head-wise decision before the gate
   uint8_t *refresh;   // [R]            final decision of the current step
   double *drift;      // [R]
@@ -63,8 +64,6 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   off += align256(sizeof(double) * 2 * (size_t)g.R * g.nchunks * kD);
   w.mean = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * 2 * (size_t)g.R * kD);
-  w.part = reinterpret_cast<double *>(p + off);
-  off += align256(sizeof(double) * 2 * (size_t)g.R);
   w.pre = reinterpret_cast<uint8_t *>(p + off);
   off += align256((size_t)g.R);
   w.refresh = reinterpret_cast<uint8_t *>(p + off);
@@ -80,14 +79,48 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   return w;
 }
 
+constexpr int kStatusTicketWord = 8, kStatusSigWord = 10;
+
+#ifdef __CUDACC__
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may be
+// scheduled while the kernel before it on the stream drains; it must not touch that kernel's results
+// before pdl_wait().  pdl_launch_dependents() in the earlier kernel lets the later one be scheduled
+// once every CTA has issued it (or exited).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
+// Validates the shape part of a config and derives the geometry: HEART_OK or an error code.
+int make_geom(const heart_config *c, Geom *g);
+// What the block means in a workspace belong to (tensor addresses, shape, strides), never 0.
+unsigned long long block_means_signature(const Geom &g, const void *Q, const void *K);
+
 // Launchers (defined in the kernel files). Each returns the cudaError_t of its launches and
 // adds the number of kernels it launched to *launches.
 cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, const Workspace &w,
                               cudaStream_t s, int *launches);
 cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta, heart_state st,
                           double *drift_out, uint8_t *refresh_out, cudaStream_t s, int *launches);
+// expect_sig != 0: the block means were left by an earlier call; the kernels check the workspace's
+// signature against it and report HEART_ERR_DEVICE_CHECK (masks untouched) on a mismatch.
 cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
-                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches);
+                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches,
+                                unsigned long long expect_sig = 0);
 // h0/hcount select the heads [h0, h0 + hcount) of every batch entry (hcount <= 0: all heads).
 cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const void *V,
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,

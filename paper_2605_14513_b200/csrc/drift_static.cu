@@ -44,8 +44,10 @@ int heart_drift_static(const heart_config *cfg, const void *Q, const void *K, co
   if (cfg == nullptr) return HEART_ERR_INVALID;
   // Size check first, from the same accounting the caller-allocated path uses (the part of the
   // workspace that the drift kernels touch: the pooled-score area of the mask predictor lies behind it).
+  Geom geom;
+  const int shape_rc = make_geom(cfg, &geom);
+  if (shape_rc != HEART_OK) return shape_rc;  // the code heart_drift gives for this cfg
   const size_t need = heart_drift_workspace_bytes(cfg);
-  if (need == 0) return HEART_ERR_UNSUPPORTED;  // shape the library does not handle at all
   if (need > (size_t)HEART_STATIC_SCRATCH_BYTES) return HEART_ERR_TOO_LARGE;
   if (!Q || !K || !delta || !st || !st->anchor_q || !st->anchor_k || !st->has_anchor) return HEART_ERR_INVALID;
   if ((reinterpret_cast<uintptr_t>(Q) & 15u) || (reinterpret_cast<uintptr_t>(K) & 15u)) return HEART_ERR_INVALID;
@@ -59,6 +61,11 @@ int heart_drift_static(const heart_config *cfg, const void *Q, const void *K, co
   if (!full.mask_bits) full.mask_bits = reinterpret_cast<uint32_t *>(scratch);
   if (!full.kv_idx) full.kv_idx = reinterpret_cast<int32_t *>(scratch);
   if (!full.kv_cnt) full.kv_cnt = reinterpret_cast<int32_t *>(scratch);
+  // The one word the kernels expect at zero (the gate's ticket counter): an earlier pair of calls that
+  // overlapped on the GPU may have left it anywhere, and the caller has no handle on this array.
+  e = cudaMemsetAsync(static_cast<int32_t *>(scratch) + kStatusTicketWord, 0, sizeof(int32_t),
+                      static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return HEART_ERR_CUDA;
   return heart_drift(cfg, Q, K, delta, &full, drift_out, refresh_out, scratch, stream);
 }
 

@@ -22,8 +22,10 @@ int cuda_fail(cudaError_t e, const char *where) {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+}  // namespace
+
 // Validates the shape part of a config and derives the geometry. Returns HEART_OK or an error.
-int make_geom(const heart_config *c, Geom *g) {
+int heart::make_geom(const heart_config *c, Geom *g) {
   if (c == nullptr) return HEART_ERR_INVALID;
   if (c->B <= 0 || c->H <= 0 || c->N <= 0) return HEART_ERR_INVALID;
   if (c->D != kD) return HEART_ERR_UNSUPPORTED;
@@ -57,6 +59,8 @@ int make_geom(const heart_config *c, Geom *g) {
   set_chunks(*g);
   return HEART_OK;
 }
+
+namespace {
 
 bool state_ok(const heart_state *st) {
   return st && st->anchor_q && st->anchor_k && st->has_anchor && st->mask_bits && st->kv_idx && st->kv_cnt;
@@ -128,9 +132,17 @@ int heart_predict_mask(const heart_config *cfg, const void *Q, const void *K, co
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   Workspace w = carve(g, workspace);
   g_launches = 0;
-  cudaError_t e = launch_block_sums(g, Q, K, w, s, &g_launches);
-  if (e != cudaSuccess) return cuda_fail(e, "block_sums");
-  e = launch_predict_mask(g, w, tau, refresh, *st, s, &g_launches);
+  cudaError_t e;
+  unsigned long long expect_sig = 0;
+  if (g.flags & HEART_BLOCK_MEANS_VALID) {
+    // the caller vouches that a heart_drift (or heart_predict_mask) on these very tensors left the block
+    // means in this workspace: no second pass over Q and K; the kernels verify the workspace's signature
+    expect_sig = block_means_signature(g, Q, K);
+  } else {
+    e = launch_block_sums(g, Q, K, w, s, &g_launches);
+    if (e != cudaSuccess) return cuda_fail(e, "block_sums");
+  }
+  e = launch_predict_mask(g, w, tau, refresh, *st, s, &g_launches, expect_sig);
   if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
   return HEART_OK;
 }
@@ -317,8 +329,10 @@ int heart_full_token_drift(const heart_config *cfg, const void *Qa, const void *
   const size_t need = (size_t)g.R * token_drift_chunks(g, &rows);  // partials live in the block-sum area
   if (need > 2 * (size_t)g.R * g.nb * kD) return HEART_ERR_INVALID;
   g_launches = 0;
-  cudaError_t e = launch_token_drift(g, Qa, Ka, Qb, Kb, w.bmean, drift_out,
-                                     static_cast<cudaStream_t>(stream), &g_launches);
+  // the partials overwrite the block means: the workspace no longer holds any
+  cudaError_t e = cudaMemsetAsync(w.status + kStatusSigWord, 0, 8, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e, "token_drift");
+  e = launch_token_drift(g, Qa, Ka, Qb, Kb, w.bmean, drift_out, static_cast<cudaStream_t>(stream), &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "token_drift");
   return HEART_OK;
 }

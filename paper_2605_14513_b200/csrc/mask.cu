@@ -82,8 +82,17 @@ __device__ __forceinline__ void cp_async_wait() {
 __global__ void __launch_bounds__(256, 2) pooled_scores_kernel(const double *__restrict__ bmean, int R, int nb,
                                                                int pitch, double scale,
                                                                const uint8_t *__restrict__ refresh,
-                                                               double *__restrict__ scores) {
+                                                               double *__restrict__ scores,
+                                                               int32_t *__restrict__ status,
+                                                               unsigned long long expect_sig) {
   const int r = blockIdx.z;
+  pdl_wait();  // refresh flags and block means come from the kernels before this one
+  pdl_launch_dependents();
+  if (expect_sig != 0 && *reinterpret_cast<const unsigned long long *>(status + kStatusSigWord) != expect_sig) {
+    // the caller vouched for block means that this workspace does not hold: report, predict nothing
+    if (threadIdx.x == 0) atomicExch(status, HEART_ERR_DEVICE_CHECK);
+    return;
+  }
   if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: nothing to predict
   const int I0 = blockIdx.y * SI, J0 = blockIdx.x * SJ;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -154,8 +163,12 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
                                                                  unsigned flags, uint32_t *__restrict__ mask_bits,
                                                                  int32_t *__restrict__ kv_idx,
                                                                  int32_t *__restrict__ kv_cnt, int idx_stride,
-                                                                 int W) {
+                                                                 int W, const int32_t *__restrict__ status,
+                                                                 unsigned long long expect_sig) {
   const int r = blockIdx.y;
+  pdl_wait();  // the scores come from the kernel before this one
+  if (expect_sig != 0 && *reinterpret_cast<const unsigned long long *>(status + kStatusSigWord) != expect_sig)
+    return;  // reported by the score kernel
   if (refresh != nullptr && refresh[r] == 0) return;  // reuse branch of Algorithm 1: mask untouched
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   extern __shared__ __align__(16) unsigned char smem_top[];
@@ -192,7 +205,9 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
     // with tau * z instead of dividing the row by z: the same ranking, the same ties and the same
     // cumulative-mass test up to rounding, at 1/3 fewer fp64 instructions per block.
     const double tau_r = (flags & HEART_FORCE_DENSE) ? 1.0 : tau[r];
-    const double t = tau_r * z;
+    // tau <= 0: every prefix reaches it, so the minimal one is the single largest block (lowest index
+    // on ties): the smallest positive threshold gives exactly that
+    const double t = (tau_r > 0.0 ? tau_r : 2.2250738585072014e-308) * z;
     const bool keep_all = !(tau_r < 1.0) || !(z >= t);
     long long theta = 0;
     int m_ties = 0, n_ties = 0;
@@ -361,31 +376,32 @@ __global__ void __launch_bounds__(32 * kRowsPerCta) top_p_kernel(const double *_
 
 template <int NJ>
 static cudaError_t launch_nj(const Geom &g, const Workspace &w, const double *tau, const uint8_t *refresh,
-                             heart_state st, int pitch, cudaStream_t s) {
+                             heart_state st, int pitch, cudaStream_t s, unsigned long long expect_sig) {
   dim3 grid((g.nb + kRowsPerCta - 1) / kRowsPerCta, g.R);
   const size_t smem = sizeof(double) * kRowsPerCta * NJ * 32;
   cudaError_t e = cudaFuncSetAttribute(top_p_kernel<NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  top_p_kernel<NJ><<<grid, 32 * kRowsPerCta, smem, s>>>(w.scores, g.nb, pitch, tau, refresh, g.flags, st.mask_bits,
-                                                     st.kv_idx, st.kv_cnt, g.idx_stride, g.W);
-  return cudaGetLastError();
+  return launch_pdl(top_p_kernel<NJ>, grid, dim3(32 * kRowsPerCta), smem, s, (const double *)w.scores, g.nb, pitch, tau,
+                    refresh, g.flags, st.mask_bits, st.kv_idx, st.kv_cnt, g.idx_stride, g.W, (const int32_t *)w.status,
+                    expect_sig);
 }
 
 cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
-                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches) {
+                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches,
+                                unsigned long long expect_sig) {
   *launches += 2;
   const int nj = (g.nb + 31) / 32, pitch = nj * 32;
   const size_t smem = sizeof(double) * 2 * (SI + SJ) * KLD;
   cudaError_t e = cudaFuncSetAttribute(pooled_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((g.nb + SJ - 1) / SJ, (g.nb + SI - 1) / SI, g.R);
-  pooled_scores_kernel<<<grid, 256, smem, s>>>(w.bmean, g.R, g.nb, pitch, g.scale, refresh, w.scores);
-  e = cudaGetLastError();
+  e = launch_pdl(pooled_scores_kernel, grid, dim3(256), smem, s, (const double *)w.bmean, g.R, g.nb, pitch, g.scale,
+                 refresh, w.scores, w.status, expect_sig);
   if (e != cudaSuccess) return e;
-  if (nj <= 8) return launch_nj<8>(g, w, tau, refresh, st, pitch, s);
-  if (nj <= 16) return launch_nj<16>(g, w, tau, refresh, st, pitch, s);
-  if (nj <= 24) return launch_nj<24>(g, w, tau, refresh, st, pitch, s);
-  return launch_nj<32>(g, w, tau, refresh, st, pitch, s);
+  if (nj <= 8) return launch_nj<8>(g, w, tau, refresh, st, pitch, s, expect_sig);
+  if (nj <= 16) return launch_nj<16>(g, w, tau, refresh, st, pitch, s, expect_sig);
+  if (nj <= 24) return launch_nj<24>(g, w, tau, refresh, st, pitch, s, expect_sig);
+  return launch_nj<32>(g, w, tau, refresh, st, pitch, s, expect_sig);
 }
 
 }  // namespace heart

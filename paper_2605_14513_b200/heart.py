@@ -16,7 +16,7 @@ _LIB_PATH = os.environ.get("HEART_LIB") or os.path.join(_HERE, "libheart.so")
 
 OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
 STATIC_SCRATCH_BYTES = 16 << 20
-FORCE_REFRESH, FORCE_DENSE = 1, 2
+FORCE_REFRESH, FORCE_DENSE, BLOCK_MEANS_VALID, ESTIMATOR_ANTIDIAG = 1, 2, 4, 8
 MAX_BLOCKS = 1024
 
 # Every symbol include/heart.h declares.
@@ -103,6 +103,12 @@ def _check(rc):
         raise HeartError(rc)
 
 
+def _with_flags(cfg, flags):
+    c = Config.from_buffer_copy(cfg)
+    c.flags = flags
+    return c
+
+
 def n_blocks(N, block):
     return (N + block - 1) // block
 
@@ -171,7 +177,11 @@ def heart_drift(cfg, Q, K, delta, st: State, ws, drift_out=None, refresh_out=Non
                              _ptr(refresh_out), _ptr(ws), _stream()))
 
 
-def heart_predict_mask(cfg, Q, K, tau, st: State, ws, refresh=None):
+def heart_predict_mask(cfg, Q, K, tau, st: State, ws, refresh=None, means_valid=False):
+    """means_valid: pass HEART_BLOCK_MEANS_VALID for this call (heart_drift has just run on the same
+    Q, K and workspace), so the pass over Q and K is not repeated."""
+    if means_valid:
+        cfg = _with_flags(cfg, cfg.flags | BLOCK_MEANS_VALID)
     _check(lib().heart_predict_mask(C.byref(cfg), _ptr(Q), _ptr(K), _ptr(tau), _ptr(refresh), C.byref(st.struct),
                                     _ptr(ws), _stream()))
 

@@ -38,8 +38,9 @@ def check_decisions(drift_gpu, refresh_gpu, drift_ref, refresh_ref, delta):
 
 def check_masks(gpu_state, ref_state, heads, tau, probs_row_fn):
     """Bit masks / lists / counts of `heads` identical, except rows whose cumulative mass sits within
-    MASS_BAND of tau or whose boundary blocks are tied to within 1e-5 relative (judged with the
-    oracle's fp64 probabilities).  Returns the number of exempted rows."""
+    MASS_BAND of tau, or whose swapped boundary blocks are tied to within 1e-5 relative AND whose
+    retained mass equals the oracle's within MASS_BAND (judged with the oracle's fp64 probabilities).
+    Returns the number of exempted rows."""
     gb, rb = mask_bits_u32(gpu_state.mask_bits), ref_state.mask_bits
     gc, rc = to_np(gpu_state.kv_cnt), ref_state.kv_cnt
     gi, ri = to_np(gpu_state.kv_idx), ref_state.kv_idx
@@ -66,10 +67,11 @@ def check_masks(gpu_state, ref_state, heads, tau, probs_row_fn):
             pmin = min(P[j] for j in G)
             p_edge = min(P[j] for j in Rf)
             assert mass >= t - MASS_BAND and mass - pmin < t + MASS_BAND, (r, I, mass, t)
+            mass_ref = sum(P[x] for x in Rf)
             for j in G ^ Rf:
-                assert abs(P[j] - p_edge) <= 1e-6 * P.max() + 1e-5 * p_edge or \
-                    abs(sum(P[x] for x in Rf) - t) <= MASS_BAND or \
-                    abs(sum(P[x] for x in Rf) - p_edge - t) <= MASS_BAND, (r, I, j, P[j], p_edge)
+                tied = abs(P[j] - p_edge) <= 1e-6 * P.max() + 1e-5 * p_edge and abs(mass - mass_ref) <= MASS_BAND
+                assert tied or abs(mass_ref - t) <= MASS_BAND or \
+                    abs(mass_ref - p_edge - t) <= MASS_BAND, (r, I, j, P[j], p_edge)
             exempt += 1
     return exempt
 

@@ -129,7 +129,9 @@ def test_step_equals_three_calls_and_checkpoint(heart, oracle):
         d2 = torch.empty(wl.R, dtype=torch.float64, device="cuda")
         r2 = torch.empty(wl.R, dtype=torch.uint8, device="cuda")
         heart.heart_drift(b.cfg, b.Q, b.K, b.delta, b.gst, b.ws, drift_out=d2, refresh_out=r2)
-        heart.heart_predict_mask(b.cfg, b.Q, b.K, b.tau, b.gst, b.ws, refresh=r2)
+        # odd steps reuse the block means heart_drift left in the workspace, even steps recompute them
+        heart.heart_predict_mask(b.cfg, b.Q, b.K, b.tau, b.gst, b.ws, refresh=r2, means_valid=bool(t & 1))
+        assert heart.heart_get_status(b.ws) == 0
         O2 = torch.full_like(b.Q, float("nan"))
         heart.heart_block_sparse_attn(b.cfg, b.Q, b.K, b.V, b.gst.kv_idx, b.gst.kv_cnt, O2, b.ws)
         assert np.array_equal(drift, to_np(d2)) and np.array_equal(refresh, to_np(r2))
@@ -200,9 +202,39 @@ def test_identical_inputs_have_exactly_zero_drift(heart, oracle):
     assert np.array_equal(d1, [0.0, 0.0]) and np.array_equal(r1, [0, 0])
 
 
+def test_block_means_valid_flag_is_checked_on_the_device(heart, oracle):
+    """HEART_BLOCK_MEANS_VALID with block means that belong to other tensors (or to none): nothing is
+    predicted, the state keeps its old masks and the status word reports the mismatch."""
+    wl = inputs.small_workload(H=2, grid=(3, 10, 14), block=64, seed=17)
+    p = Pair(wl, heart, oracle)
+    # a fresh (zeroed) workspace holds no block means at all
+    heart.heart_predict_mask(p.cfg, p.Q, p.K, p.tau, p.gst, p.ws, means_valid=True)
+    assert heart.heart_get_status(p.ws) == heart.ERR_DEVICE_CHECK
+    assert int(p.gst.kv_cnt.sum()) == 0
+    # means of (Q, K) are there after heart_drift; claiming them for another K tensor is caught
+    heart.heart_drift(p.cfg, p.Q, p.K, p.delta, p.gst, p.ws)
+    K2 = p.K.clone()
+    heart.heart_predict_mask(p.cfg, p.Q, K2, p.tau, p.gst, p.ws, means_valid=True)
+    assert heart.heart_get_status(p.ws) == heart.ERR_DEVICE_CHECK
+    assert int(p.gst.kv_cnt.sum()) == 0
+    # the honest call works and equals the recomputing call
+    heart.heart_predict_mask(p.cfg, p.Q, p.K, p.tau, p.gst, p.ws, means_valid=True)
+    assert heart.heart_get_status(p.ws) == 0
+    a = [t.clone() for t in p.gst.tensors()]
+    heart.heart_predict_mask(p.cfg, p.Q, p.K, p.tau, p.gst, p.ws)
+    for x, y in zip(a, p.gst.tensors()):
+        assert torch.equal(x, y)
+    assert int(p.gst.kv_cnt.min()) >= 1
+    # the full-token drift uses the block-mean area as scratch: the means are gone afterwards
+    d = torch.empty(wl.R, dtype=torch.float64, device="cuda")
+    heart.heart_full_token_drift(p.cfg, p.Q, p.K, p.Q, p.K, d, p.ws)
+    heart.heart_predict_mask(p.cfg, p.Q, p.K, p.tau, p.gst, p.ws, means_valid=True)
+    assert heart.heart_get_status(p.ws) == heart.ERR_DEVICE_CHECK
+
+
 # ------------------------------------------------------------------ degenerate thresholds / flags
 def test_tau_extremes_and_force_flags(heart, oracle):
-    wl = inputs.small_workload(H=3, grid=(3, 10, 14), block=64, seed=8, tau=[1.0, 1e-9, 0.5])
+    wl = inputs.small_workload(H=5, grid=(3, 10, 14), block=64, seed=8, tau=[1.0, 1e-9, 0.5, 0.0, -1.0])
     p = Pair(wl, heart, oracle)
     O, _, _, _ = p.gpu_step()
     p.oracle_step(want_O=False)
@@ -210,7 +242,9 @@ def test_tau_extremes_and_force_flags(heart, oracle):
     cnt = to_np(p.gst.kv_cnt)
     assert np.all(cnt[0] == nb)               # tau = 1 -> dense mask
     assert np.all(cnt[1] == 1)                # tau -> 0+ -> exactly one block
-    assert check_masks(p.gst, p.ost, range(3), wl.tau, p.probs_row) == 0
+    assert np.all(cnt[3] == 1) and np.all(cnt[4] == 1)  # tau <= 0: still the one largest block
+    assert np.array_equal(cnt, p.ost.kv_cnt)
+    assert check_masks(p.gst, p.ost, range(5), wl.tau, p.probs_row) == 0
     # dense warm-up step: state untouched, output = dense attention
     before = [t.clone() for t in p.gst.tensors()]
     O, lse, drift, refresh = p.gpu_step(flags=heart.FORCE_DENSE)
