@@ -1,16 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the HEART layer-step (drift + mask prediction + block-sparse attention) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload wan1.3b-480p] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload hunyuan-720p] [--impl reference]
 
 A "step" is one heart_step call = one whole pass of the hot path over one denoising step of
 synthetic Q/K/V (seeded, shaped like the paper's Wan2.1 / HunyuanVideo activations), with the TMR
 state carried from step to step so refresh and reuse mix as in a real sweep.  Prints ONE JSON line.
 
+The headline workload is the largest single-GPU configuration (hunyuan-720p: 24 heads, 118 800
+tokens, block 128, every head refreshing at every step); the other four configurations are measured
+in the same run on a few steps each and reported in `per_workload`, each with its own clock record.
+
 The path does not shard (one layer's heads could be split across GPUs with no exchange, but the
-north star is a single-GPU kernel library): with --gpus N every rank runs an independent replica
+library is a single-GPU kernel library): with --gpus N every rank runs an independent replica
 ("replicas only"), and `value` is the time per layer-step of the whole job = max-over-ranks step
-time / N.
+time / N.  Run without torchrun, --gpus N starts the N ranks itself.
 
 --impl reference times the CPU oracle (oracle/) as it stands on the host cores, on a bounded
 sample of the same workload, and prints the same line with "impl": "reference".
@@ -18,6 +22,7 @@ sample of the same workload, and prints the same line with "impl": "reference".
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -29,6 +34,9 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "ms per layer-step (drift+mask+attn)"
+HEADLINE = "hunyuan-720p"
+OTHERS = ("tiny", "wan1.3b-480p", "wan14b-480p", "wan14b-720p")
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "attn_tc_kernel_dram_traffic.txt")
 
 
 def parse():
@@ -36,11 +44,13 @@ def parse():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="wan1.3b-480p")
+    ap.add_argument("--workload", default=HEADLINE)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cpu-sample-rows", type=int, default=384, help="query blocks the CPU oracle attends per step")
+    ap.add_argument("--cpu-sample-rows", type=int, default=0,
+                    help="query blocks the CPU oracle attends per step (0: sized for about a second per step)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-per-workload", action="store_true", help="measure the headline workload only")
     return ap.parse_args()
 
 
@@ -51,6 +61,25 @@ def peaks():
         return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
                 "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def dram_traffic(workload):
+    """DRAM bytes per attention launch (ncu, dram__bytes_read.sum + dram__bytes_write.sum) from the table
+    under profiles/ that the captures are summarised into; None where no capture exists."""
+    try:
+        for line in open(TRAFFIC_TABLE):
+            f = line.split()
+            if len(f) >= 2 and not line.startswith("#") and f[0] == workload:
+                return float(f[1])
+    except OSError:
+        pass
+    return None
+
+
+def config_of(wl):
+    """The workload description both arms print (identical in both)."""
+    return {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "grid": list(wl.grid), "D": wl.D,
+            "block": wl.block, "n_blocks": wl.n_blocks, "pos_scale": float(wl.pos_scale[0]), "seed": wl.seed}
 
 
 class ClockSampler:
@@ -141,25 +170,32 @@ def retained_flops(torch, st, wl):
     return 4.0 * wl.D * (keys * qrows[None, :]).sum(), cnt.sum()
 
 
-def run_ours(args, rank, world):
-    import numpy as np
-    import torch
-    import torch.distributed as dist
+def attention_roofline(pk, tflops, clocks, region_ms, flops_step, ms_attn, traffic):
+    """The attention fraction against both measured cuBLAS peaks, and which of the two applies to this
+    run: the sustained one when the clock record shows the power cap (or the timed region lasted
+    seconds), the burst one when the SM clock sat at its maximum for a region of milliseconds."""
+    capped = bool(clocks) and "sw_power_cap" in (clocks.get("reasons") or [])
+    long_region = region_ms >= 1000.0
+    which = "sustained" if (capped or long_region) else "burst"
+    peak = pk["bf16_tflops_sustained"] if which == "sustained" else pk["bf16_tflops"]
+    why = ("sw_power_cap active during the timed passes" if capped else
+           "timed region of %.0f ms" % region_ms if long_region else
+           "SM clock at its maximum with no throttle reason, region of %.0f ms" % region_ms)
+    return {"kernel": "block-sparse attention", "bound": "tensor", "achieved": tflops, "peak": peak,
+            "unit": "TFLOP/s", "frac": tflops / peak, "traffic": traffic,
+            "peak_source": f"{pk['source']} cuBLAS bf16, {which} figure ({why})",
+            "frac_of_burst_peak": tflops / pk["bf16_tflops"], "burst_peak": pk["bf16_tflops"],
+            "frac_of_sustained_peak": tflops / pk["bf16_tflops_sustained"],
+            "sustained_peak": pk["bf16_tflops_sustained"],
+            "arithmetic": "%.4g flop per launch / %.4f ms = %.1f TFLOP/s; / %.1f = %.3f" % (
+                flops_step, ms_attn, tflops, peak, tflops / peak),
+            "flops_per_launch": flops_step, "ms_per_launch": ms_attn}
 
-    from paper_2605_14513_b200 import heart, inputs, replicas
 
-    heart.lib()  # fails loudly if the CUDA library is missing
-    local = int(os.environ.get("LOCAL_RANK", 0))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    pk = peaks()
-    wl = inputs.workload(args.workload)
-    K, W = args.steps, args.warmup
+def measure(torch, heart, inputs, replicas, wl, K, W, dev, pk, rank, sampler_uuid, full):
+    """W warm-up + K timed heart_step calls on device-resident inputs, then the per-stage, accounting,
+    back-to-back and (where it fits in time) dense passes.  Returns (record, context for e2e/cpu)."""
     n_inputs = K + W
-
-    # ---- synthetic inputs, all resident in HBM before anything is timed
     seq = inputs.Sequence(wl, dev)
     steps_in = []
     for t in range(n_inputs):
@@ -186,50 +222,49 @@ def run_ours(args, rank, world):
     for t in range(W):
         step(t)
     torch.cuda.synchronize()
-    ckpt = st.state_dict()  # state after warm-up: the e2e and per-stage passes restart from here
+    ckpt = st.state_dict()  # state after warm-up: the later passes restart from here
 
-    # ---- timed region: exactly K steps, device-resident inputs, one event pair per step
-    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", "")
-    sampler = ClockSampler(uuid) if rank == 0 else None
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    # ---- timed region: exactly K steps, device-resident inputs
+    sampler = ClockSampler(sampler_uuid) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches = 0
     barrier()
     t_wall = time.perf_counter()
+    e0.record()
     for k in range(K):
-        ev[k][0].record()
         step(W + k)
-        ev[k][1].record()
         launches += heart.heart_last_launch_count()
+    e1.record()
     barrier()
     wall_ms = (time.perf_counter() - t_wall) * 1e3
     clocks = sampler.stop() if sampler else None
-    total_ms = ev[0][0].elapsed_time(ev[-1][1])
+    total_ms = e0.elapsed_time(e1)
     assert heart.heart_get_status(ws) == 0
     total_ms = replicas.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / K
 
     # ---- per-stage pass: the same K steps as three C-ABI calls, one event pair per call.  Nothing here
-    # synchronises with the host, and nothing but the three calls and the event records is enqueued (the
-    # accounting kernels of the pass after it would otherwise sit between a step's attention and the next
-    # step's drift call and stretch the latter's interval by ~14 us).
+    # synchronises with the host, and nothing but the three calls and the event records is enqueued.  The
+    # mask call reuses the block means that the drift call has just left in the workspace.
     st.load_state_dict(ckpt)
     stage_ev = []
     r2 = torch.empty_like(refresh)
     torch.cuda.synchronize()
-    sampler2 = ClockSampler(uuid) if rank == 0 else None  # this pass has its own clock record
+    sampler2 = ClockSampler(sampler_uuid) if rank == 0 else None  # this pass has its own clock record
     for k in range(K):
         Q, Kt, V = steps_in[W + k]
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         e[0].record()
         heart.heart_drift(cfg, Q, Kt, delta, st, ws, refresh_out=r2)
         e[1].record()
-        heart.heart_predict_mask(cfg, Q, Kt, tau, st, ws, refresh=r2)
+        heart.heart_predict_mask(cfg, Q, Kt, tau, st, ws, refresh=r2, means_valid=True)
         e[2].record()
         heart.heart_block_sparse_attn(cfg, Q, Kt, V, st.kv_idx, st.kv_cnt, O, ws)
         e[3].record()
         stage_ev.append(e)
     torch.cuda.synchronize()
     clocks_stage = sampler2.stop() if sampler2 else None
+    assert heart.heart_get_status(ws) == 0
     # ---- accounting pass (untimed): the same decisions and masks again from the same state; the flop /
     # pair / refresh counts are accumulated on the device.
     st.load_state_dict(ckpt)
@@ -237,7 +272,7 @@ def run_ours(args, rank, world):
     for k in range(K):
         Q, Kt, V = steps_in[W + k]
         heart.heart_drift(cfg, Q, Kt, delta, st, ws, refresh_out=r2)
-        heart.heart_predict_mask(cfg, Q, Kt, tau, st, ws, refresh=r2)
+        heart.heart_predict_mask(cfg, Q, Kt, tau, st, ws, refresh=r2, means_valid=True)
         f, p = retained_flops(torch, st, wl)
         acc += torch.stack([f, p, r2.sum().to(torch.float64)])
     torch.cuda.synchronize()
@@ -251,9 +286,21 @@ def run_ours(args, rank, world):
     attn_tflops = flops_step / (ms_attn * 1e-3) / 1e12
     stats_bytes = 4.0 * wl.R * wl.N * wl.D  # Q and K read once (bf16)
 
-    # ---- the attention kernel alone, back to back on the masks of the last step (each launch on another
-    # step's Q/K/V, so nothing is L2-warm): reported beside the per-stage figure, which reads a few percent
-    # longer because every launch there follows the mask kernels of its own step
+    # ---- back-to-back passes: each kernel family alone, every launch on another step's tensors (nothing is
+    # L2-warm).  Inside a step the drift call follows the attention kernel, whose output is still being
+    # written back from L2, and reads a few microseconds longer; both figures are reported.
+    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    st_b2b = heart.State(cfg, dev)
+    st_b2b.load_state_dict(ckpt)
+    torch.cuda.synchronize()
+    a0.record()
+    for k in range(K):
+        Q, Kt, V = steps_in[W + k]
+        heart.heart_drift(cfg, Q, Kt, delta, st_b2b, ws)
+    a1.record()
+    torch.cuda.synchronize()
+    ms_drift_b2b = a0.elapsed_time(a1) / K
+    del st_b2b
     f_last, _ = retained_flops(torch, st, wl)
     a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a0.record()
@@ -268,7 +315,7 @@ def run_ours(args, rank, world):
     # ---- the same attention kernel with a full mask, measured where it fits in time (a dense run of the
     # two 720P shapes would take 0.1-0.15 s per launch): the sparse path's speedup over its own dense mode
     dense_ms = None
-    if dense_flops < 3e13:
+    if dense_flops < 3e13 and full:
         cfg_dense = heart.make_config(wl.B, wl.H, wl.N, wl.block, flags=heart.FORCE_DENSE)
         Q, Kt, V = steps_in[W]
         heart.heart_block_sparse_attn(cfg_dense, Q, Kt, V, None, None, O, ws)
@@ -280,73 +327,158 @@ def run_ours(args, rank, world):
         torch.cuda.synchronize()
         dense_ms = a.elapsed_time(b_) / 3
 
-    # ---- end-to-end pass: host (pinned) Q/K/V in, O/drift/refresh out, through heart_step_host
-    e2e = None
-    if not args.no_e2e:
-        Ke = min(K, max(1, int(6e9 // (4 * 2 * wl.R * wl.N * wl.D))))  # cap pinned memory at ~6 GB
-        host_in = [tuple(x.cpu().pin_memory() for x in steps_in[W + k]) for k in range(Ke)]
-        Oh = torch.empty(O.shape, dtype=O.dtype).pin_memory()
-        dh = torch.empty(wl.R, dtype=torch.float64).pin_memory()
-        rh = torch.empty(wl.R, dtype=torch.uint8).pin_memory()
-        staging = tuple(torch.empty_like(O) for _ in range(4))
-        st.load_state_dict(ckpt)
-        heart.heart_step_host(cfg, *host_in[0], delta, tau, st, Oh, staging, ws, drift_host=dh, refresh_host=rh)
-        st.load_state_dict(ckpt)
-        barrier()
-        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for k in range(Ke):
-            heart.heart_step_host(cfg, *host_in[k], delta, tau, st, Oh, staging, ws, drift_host=dh, refresh_host=rh)
-        b_.record()
-        barrier()
-        e2e_ms = a.elapsed_time(b_) / Ke
-        e2e_ms = replicas.max_over_ranks(e2e_ms, dev)
-        tensor_bytes = 2 * wl.R * wl.N * wl.D
-        e2e = {"value": replicas.job_ms_per_layer_step(e2e_ms, world), "unit": "ms", "steps": Ke, "h2d_bytes_per_step": 3 * tensor_bytes,
-               "d2h_bytes_per_step": tensor_bytes + 9 * wl.R,
-               "api": "heart_step_host (pinned host Q/K/V in, O + drift + refresh out)"}
-        del host_in, staging
+    hbm = stats_bytes / (ms_drift * 1e-3) / 1e9
+    hbm_b2b = stats_bytes / (ms_drift_b2b * 1e-3) / 1e9
+    l2_note = ("inputs larger than L2 (every step reads new Q/K/V tensors, >= 3x the 126 MB L2)"
+               if 6 * wl.R * wl.N * wl.D > 126e6 else "L2-resident (tiny case): not a roofline number")
+    region_ms = (ms_drift + ms_mask + ms_attn) * K
+    rec = {
+        "workload": wl.name, "config": config_of(wl), "steps": K, "warmup": W, "ms_per_step": ms_per_step,
+        "l2": l2_note,
+        "stages_ms": {"drift": ms_drift, "mask": ms_mask, "attention": ms_attn,
+                      "sum_of_separate_calls": ms_drift + ms_mask + ms_attn},
+        "density": density, "refresh_rate": refreshed / (K * wl.R),
+        "retained_tflops": attn_tflops,
+        "dense_equivalent_tflops": dense_flops / (ms_attn * 1e-3) / 1e12,
+        "dense_equivalent_speedup_at_same_throughput": dense_flops / flops_step,
+        "attention_ms_back_to_back": ms_attn_b2b, "retained_tflops_back_to_back": attn_tflops_b2b,
+        "dense_attention_ms_measured": dense_ms,
+        "dense_tflops_measured": (dense_flops / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
+        "attention_speedup_vs_measured_dense": (dense_ms / ms_attn) if dense_ms else None,
+        "roofline": attention_roofline(pk, attn_tflops, clocks_stage, region_ms, flops_step, ms_attn,
+                                       dram_traffic(wl.name)),
+        "roofline_stats": {"kernel": "block sums + drift (heart_drift)", "bound": "hbm", "achieved": hbm,
+                           "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm / pk["hbm_gbs"],
+                           "frac_of_nominal_8TBps": hbm / 8000.0, "bytes_per_launch": stats_bytes,
+                           "ms_per_launch": ms_drift, "peak_source": pk["source"] + " copy bandwidth",
+                           "back_to_back": {"ms_per_launch": ms_drift_b2b, "achieved": hbm_b2b,
+                                            "frac": hbm_b2b / pk["hbm_gbs"]}},
+        "gpu_launches": launches, "wall_ms_timed_region": wall_ms, "clocks": clocks,
+        "clocks_stage_pass": clocks_stage,
+    }
+    ctx = dict(wl=wl, steps_in=steps_in, W=W, K=K, cfg=cfg, st=st, ws=ws, ckpt=ckpt, delta=delta, tau=tau, O=O,
+               barrier=barrier)
+    return rec, ctx
+
+
+def measure_e2e(torch, heart, replicas, ctx, dev, world):
+    """Host (pinned) Q/K/V in, O/drift/refresh out, through heart_step_host."""
+    wl, steps_in, W, K = ctx["wl"], ctx["steps_in"], ctx["W"], ctx["K"]
+    cfg, st, ws, O = ctx["cfg"], ctx["st"], ctx["ws"], ctx["O"]
+    Ke = min(K, max(1, int(6e9 // (4 * 2 * wl.R * wl.N * wl.D))))  # cap pinned memory at ~6 GB
+    host_in = [tuple(x.cpu().pin_memory() for x in steps_in[W + k]) for k in range(Ke)]
+    Oh = torch.empty(O.shape, dtype=O.dtype).pin_memory()
+    dh = torch.empty(wl.R, dtype=torch.float64).pin_memory()
+    rh = torch.empty(wl.R, dtype=torch.uint8).pin_memory()
+    staging = tuple(torch.empty_like(O) for _ in range(4))
+    st.load_state_dict(ctx["ckpt"])
+    heart.heart_step_host(cfg, *host_in[0], ctx["delta"], ctx["tau"], st, Oh, staging, ws, drift_host=dh, refresh_host=rh)
+    st.load_state_dict(ctx["ckpt"])
+    ctx["barrier"]()
+    a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for k in range(Ke):
+        heart.heart_step_host(cfg, *host_in[k], ctx["delta"], ctx["tau"], st, Oh, staging, ws, drift_host=dh, refresh_host=rh)
+    b_.record()
+    ctx["barrier"]()
+    e2e_ms = replicas.max_over_ranks(a.elapsed_time(b_) / Ke, dev)
+    tensor_bytes = 2 * wl.R * wl.N * wl.D
+    return {"value": replicas.job_ms_per_layer_step(e2e_ms, world), "unit": "ms", "steps": Ke,
+            "h2d_bytes_per_step": 3 * tensor_bytes, "d2h_bytes_per_step": tensor_bytes + 9 * wl.R,
+            "api": "heart_step_host (pinned host Q/K/V in, O + drift + refresh out)"}
+
+
+def run_ours(args, rank, world):
+    import gc
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_14513_b200 import heart, inputs, replicas
+
+    heart.lib()  # fails loudly if the CUDA library is missing
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    pk = peaks()
+    wl = inputs.workload(args.workload)
+    K, W = args.steps, args.warmup
+    uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", "")
+
+    rec, ctx = measure(torch, heart, inputs, replicas, wl, K, W, dev, pk, rank, uuid, full=True)
+    e2e = None if args.no_e2e else measure_e2e(torch, heart, replicas, ctx, dev, world)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline(args, ctx["wl"], ctx["steps_in"], ctx["W"])
+    del ctx
+    gc.collect()
+    torch.cuda.empty_cache()
+
+    per = []
+    if not args.no_per_workload and world == 1:
+        names = [n for n in OTHERS + (HEADLINE,) if n != wl.name]
+        for name in names:
+            w2 = inputs.workload(name)
+            k2 = min(K, 2 if w2.name == "tiny" else 6)
+            r2, c2 = measure(torch, heart, inputs, replicas, w2, k2, 3, dev, pk, rank, uuid, full=False)
+            del c2
+            gc.collect()
+            torch.cuda.empty_cache()
+            per.append(r2)
+        # the configuration text taken literally (positional scale 0.5): 83-98 % of the blocks are retained at
+        # these thresholds, so the sparse path degenerates to near-dense attention; a secondary record
+        lit = inputs.workload("wan1.3b-480p-literal")
+        r2, c2 = measure(torch, heart, inputs, replicas, lit, min(K, 4), 3, dev, pk, rank, uuid, full=False)
+        del c2
+        gc.collect()
+        torch.cuda.empty_cache()
+        per.append(r2)
 
     out = None
     if rank == 0:
-        peak_tf = pk["bf16_tflops_sustained"]
-        # DRAM bytes per attention launch from the ncu capture summarised in profiles/ (this workload only)
-        traffic = {"wan1.3b-480p": 399.1e6}.get(wl.name)
-        roofline = {"kernel": "block-sparse attention", "bound": "tensor", "achieved": attn_tflops, "peak": peak_tf,
-                    "unit": "TFLOP/s", "frac": attn_tflops / peak_tf, "traffic": traffic,
-                    "peak_source": pk["source"] + " (sustained bf16 cuBLAS, kernel timed inside a long step)",
-                    "flops_per_launch": flops_step, "ms_per_launch": ms_attn}
-        hbm = stats_bytes / (ms_drift * 1e-3) / 1e9
         out = {
-            "metric": METRIC, "value": replicas.job_ms_per_layer_step(ms_per_step, world), "unit": "ms", "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "grid": list(wl.grid), "D": wl.D,
-                       "block": wl.block, "n_blocks": wl.n_blocks, "parallelism": "replicas only" if world > 1 else "1 gpu",
-                       "l2": "inputs larger than L2 (every step reads new Q/K/V tensors, >= 3x the 126 MB L2)"
-                       if 6 * wl.R * wl.N * wl.D > 126e6 else "L2-resident (tiny case): not a roofline number"},
-            "stages_ms": {"drift": ms_drift, "mask": ms_mask, "attention": ms_attn,
-                          "sum_of_separate_calls": ms_drift + ms_mask + ms_attn},
-            "density": density, "refresh_rate": refreshed / (K * wl.R),
-            "retained_tflops": attn_tflops, "retained_tflops_vs_bf16_peak": attn_tflops / pk["bf16_tflops"],
-            "dense_equivalent_tflops": dense_flops / (ms_attn * 1e-3) / 1e12,
-            "dense_equivalent_speedup_at_same_throughput": dense_flops / flops_step,
-            "attention_ms_back_to_back": ms_attn_b2b, "retained_tflops_back_to_back": attn_tflops_b2b,
-            "dense_attention_ms_measured": dense_ms,
-            "dense_tflops_measured": (dense_flops / (dense_ms * 1e-3) / 1e12) if dense_ms else None,
-            "attention_speedup_vs_measured_dense": (dense_ms / ms_attn) if dense_ms else None,
-            "roofline": roofline,
-            "roofline_stats": {"kernel": "block sums + drift (heart_drift)", "bound": "hbm", "achieved": hbm,
-                               "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": hbm / pk["hbm_gbs"],
-                               "frac_of_nominal_8TBps": hbm / 8000.0, "bytes_per_launch": stats_bytes,
-                               "ms_per_launch": ms_drift},
-            "gpu_launches": launches, "wall_ms_timed_region": wall_ms, "clocks": clocks,
-            "clocks_stage_pass": clocks_stage, "e2e": e2e,
+            "metric": METRIC, "value": replicas.job_ms_per_layer_step(rec["ms_per_step"], world), "unit": "ms",
+            "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": rec["ms_per_step"], "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": rec["config"], "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": rec["l2"],
         }
-    return out, (wl, steps_in, W)
+        for k in ("stages_ms", "density", "refresh_rate", "retained_tflops", "dense_equivalent_tflops",
+                  "dense_equivalent_speedup_at_same_throughput", "attention_ms_back_to_back",
+                  "retained_tflops_back_to_back", "dense_attention_ms_measured", "dense_tflops_measured",
+                  "attention_speedup_vs_measured_dense", "roofline", "roofline_stats", "gpu_launches",
+                  "wall_ms_timed_region", "clocks", "clocks_stage_pass"):
+            out[k] = rec[k]
+        out["e2e"] = e2e
+        if cpu is not None:
+            out["cpu_baseline"] = cpu
+        out["per_workload"] = [
+            {"workload": r["workload"], "config": r["config"], "steps": r["steps"], "ms_per_step": r["ms_per_step"],
+             "stages_ms": r["stages_ms"], "density": r["density"], "refresh_rate": r["refresh_rate"],
+             "retained_tflops": r["retained_tflops"], "retained_tflops_back_to_back": r["retained_tflops_back_to_back"],
+             "attention_frac": r["roofline"]["frac"], "attention_frac_of_burst_peak": r["roofline"]["frac_of_burst_peak"],
+             "attention_frac_of_sustained_peak": r["roofline"]["frac_of_sustained_peak"],
+             "attention_peak_used": r["roofline"]["peak_source"], "attention_dram_traffic": r["roofline"]["traffic"],
+             "heart_drift_frac": r["roofline_stats"]["frac"],
+             "heart_drift_frac_back_to_back": r["roofline_stats"]["back_to_back"]["frac"],
+             "l2": r["l2"], "clocks": r["clocks"], "clocks_stage_pass": r["clocks_stage_pass"]} for r in per]
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return out
 
 
-def oracle_sample_step(oracle, inputs, np, wl, ost, Qb, Kb, Vb, rs, n_rows):
+def sample_rows_for(wl, requested):
+    """Query blocks the oracle attends per step: about a second of CPU work on ~16 cores."""
+    if requested > 0:
+        return requested
+    keys_per_row = 0.12 * wl.n_blocks * wl.block  # ~12 % density
+    flop_per_row = 4.0 * wl.block * keys_per_row * wl.D
+    return int(max(8, min(384, 3.0e10 // flop_per_row)))
+
+
+def oracle_sample_step(oracle, np, wl, ost, Qb, Kb, Vb, rs, n_rows):
     """One oracle layer-step on a bounded sample: drift + decision + masks in full, attention on
     n_rows query blocks, its time scaled by retained pairs.  Returns (seconds extrapolated, seconds spent)."""
     t0 = time.perf_counter()
@@ -362,8 +494,11 @@ def oracle_sample_step(oracle, inputs, np, wl, ost, Qb, Kb, Vb, rs, n_rows):
 
 
 def run_reference(args):
-    """The oracle as it stands, on the host cores (rank 0 only)."""
+    """The oracle as it stands, on the host cores (rank 0 only).  The synthetic inputs are generated
+    on the GPU when there is one (the generator is shared by both arms and is not timed), else on the
+    CPU; everything timed is the oracle on the host."""
     import numpy as np
+    import torch
 
     from oracle import heart_oracle as oracle
     from paper_2605_14513_b200 import inputs
@@ -371,13 +506,15 @@ def run_reference(args):
     oracle.build()
     wl = inputs.workload(args.workload)
     K, W = args.steps, args.warmup
-    seq = inputs.Sequence(wl, "cpu")
+    gen_dev = "cuda" if torch.cuda.is_available() else "cpu"
+    seq = inputs.Sequence(wl, gen_dev)
     ost = oracle.State(wl.B, wl.H, wl.N, wl.D, wl.block)
     rs = np.random.RandomState(0)
+    n_rows = sample_rows_for(wl, args.cpu_sample_rows)
     est, spent = [], 0.0
     for t in range(W + K):
         Qb, Kb, Vb = (inputs.bits(x) for x in seq.bf16())
-        e, s = oracle_sample_step(oracle, inputs, np, wl, ost, Qb, Kb, Vb, rs, args.cpu_sample_rows)
+        e, s = oracle_sample_step(oracle, np, wl, ost, Qb, Kb, Vb, rs, n_rows)
         if t >= W:
             est.append(e)
             spent += s
@@ -385,14 +522,14 @@ def run_reference(args):
             seq.advance()
     ms = 1e3 * sum(est) / K
     cores = os.cpu_count()
-    sample = (f"per step: token means, decision and masks in full; attention on {args.cpu_sample_rows} random "
+    sample = (f"per step: token means, decision and masks in full; attention on {n_rows} random "
               f"query blocks scaled by retained pairs ({spent:.1f} s of CPU work in {K} steps)")
     return {"impl": "reference", "metric": METRIC, "value": ms, "unit": "ms", "n_gpus": args.gpus, "steps": K,
             "warmup": W, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "B": wl.B, "H": wl.H, "N": wl.N, "grid": list(wl.grid), "D": wl.D,
-                       "block": wl.block, "n_blocks": wl.n_blocks},
-            "cpu_baseline": {"value": ms, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample},
+            "dtype": "f64", "data": "synthetic", "config": config_of(wl), "extrapolated": True,
+            "cpu_seconds_spent_in_timed_steps": spent,
+            "cpu_baseline": {"value": ms, "unit": "ms", "cores": cores, "kind": "oracle", "sample": sample,
+                             "extrapolated": True},
             "e2e": {"value": ms, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
 
@@ -407,12 +544,13 @@ def cpu_baseline(args, wl, steps_in, W):
     oracle.build()
     ost = oracle.State(wl.B, wl.H, wl.N, wl.D, wl.block)
     rs = np.random.RandomState(0)
+    n_rows = sample_rows_for(wl, args.cpu_sample_rows)
     est, spent, n = [], 0.0, 0
     budget = 20.0
     # step 0 builds the anchors and masks (all heads refresh); later steps show the steady mix
     for t in range(min(len(steps_in), W + 3)):
         Qb, Kb, Vb = (inputs.bits(x) for x in steps_in[t])
-        e, s = oracle_sample_step(oracle, inputs, np, wl, ost, Qb, Kb, Vb, rs, args.cpu_sample_rows)
+        e, s = oracle_sample_step(oracle, np, wl, ost, Qb, Kb, Vb, rs, n_rows)
         spent += s
         if t >= 1:
             est.append(e)
@@ -422,31 +560,41 @@ def cpu_baseline(args, wl, steps_in, W):
     if not est:
         est = [e]
     ms = 1e3 * sum(est) / len(est)
-    return {"value": ms, "unit": "ms", "cores": os.cpu_count(), "kind": "oracle",
+    return {"value": ms, "unit": "ms", "cores": os.cpu_count(), "kind": "oracle", "extrapolated": True,
             "sample": (f"{n} steps of the same inputs ({len(est)} after the all-refresh first step averaged); per step: "
-                       f"token means, decision and masks in full, attention on {args.cpu_sample_rows} random query blocks "
+                       f"token means, decision and masks in full, attention on {n_rows} random query blocks "
                        f"scaled by retained pairs; {spent:.1f} s of CPU work")}
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` outside torchrun: start the N ranks (one process per GPU)."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
     args = parse()
     rank = int(os.environ.get("RANK", 0))
-    world = int(os.environ.get("WORLD_SIZE", 1))
     if args.impl == "reference":
         if rank == 0:
             print(json.dumps(run_reference(args)), flush=True)
-        return
-    out, (wl, steps_in, W) = run_ours(args, rank, world)
+        return 0
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        return spawn_ranks(args.gpus)
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if world != args.gpus:
+        print(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={world}: launch one rank per GPU", file=sys.stderr)
+        return 2
+    out = run_ours(args, rank, world)
     if rank == 0:
-        if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = cpu_baseline(args, wl, steps_in, W)
         print(json.dumps(out), flush=True)
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.barrier()
-        dist.destroy_process_group()
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

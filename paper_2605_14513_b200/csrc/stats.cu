@@ -174,6 +174,14 @@ __global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restri
   const int i0 = grp * per, i1 = min(nchunks, i0 + per);
   const double *src = psum + ((size_t)z * R + r) * nchunks * kD + d;
   const bool gate_on = a.gate_lo > 0.0 || a.gate_hi < 1.0;
+  // What does not come from the block-sum pass is fetched while that pass drains.
+  double anc = 0.0, dl = 0.0;
+  bool had = false;
+  if (threadIdx.x < 2 * kD) anc = ((threadIdx.x >> 7) ? a.anchor_k : a.anchor_q)[(size_t)r * kD + d];
+  if (threadIdx.x == 0) {
+    had = a.has_anchor[r] != 0;
+    dl = a.delta[r];
+  }
   pdl_wait();  // the partial sums come from the kernel before this one
   pdl_launch_dependents();
   double s = 0.0;
@@ -186,7 +194,6 @@ __global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restri
     const int zz = threadIdx.x >> 7;
     m = (((sm[zz][0][d] + sm[zz][1][d]) + sm[zz][2][d]) + sm[zz][3][d]) / (double)N;
     mean[((size_t)zz * R + r) * kD + d] = m;
-    const double anc = (zz ? a.anchor_k : a.anchor_q)[(size_t)r * kD + d];
     double v = fabs(anc - m);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);  // same tree in every lane
@@ -195,9 +202,8 @@ __global__ void __launch_bounds__(1024) mean_drift_kernel(const double *__restri
   __syncthreads();
   if (threadIdx.x == 0) {
     const double pq = (wsum[0] + wsum[1]) + (wsum[2] + wsum[3]), pk = (wsum[4] + wsum[5]) + (wsum[6] + wsum[7]);
-    const bool had = a.has_anchor[r] != 0;
     const double dr = had ? (pq + pk) : __longlong_as_double(0x7ff0000000000000LL);
-    bool rf = !had || (dr > a.delta[r]);
+    bool rf = !had || (dr > dl);
     if (a.flags & HEART_FORCE_REFRESH) rf = true;
     if (a.drift_out) a.drift_out[r] = dr;
     if (!gate_on) {

@@ -139,6 +139,12 @@ def workload(name: str) -> Workload:
         delta = np.full(H, _rw_drift(0.03, 5, N))
         return Workload(name, H, grid, 64, tau, delta, eps, np.full(H, 2.6), seed=2, steps=50,
                         note="shared delta = 5-step drift of the geometric-mid eps")
+    if name == "wan1.3b-480p-literal":
+        # the configuration text taken literally: positional term scaled 0.5 (pooled logits then span so
+        # little that 83-98 % of the blocks are retained at these thresholds); a secondary benchmark record
+        w = workload("wan1.3b-480p")
+        return Workload(name, w.H, w.grid, w.block, w.tau, w.delta, w.eps, np.full(w.H, 0.5), seed=w.seed,
+                        steps=w.steps, note="positional scale 0.5 as the configuration text says")
     if name == "wan14b-480p":
         H, grid = 40, (21, 30, 52)
         rs = np.random.RandomState(3)
