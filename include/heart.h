@@ -52,8 +52,9 @@ enum {
   HEART_ERR_CUDA = 3,         /* a CUDA call or launch failed (see heart_strerror)      */
   HEART_ERR_DEVICE_CHECK = 4, /* a device-side check failed: bad index-list entry or a  */
                               /* bounded wait ran out; only via heart_get_status        */
-  HEART_ERR_TOO_LARGE = 5     /* heart_drift_static: the shape needs more scratch than   */
+  HEART_ERR_TOO_LARGE = 5,    /* heart_drift_static: the shape needs more scratch than   */
                               /* HEART_STATIC_SCRATCH_BYTES                              */
+  HEART_ERR_INFEASIBLE = 6    /* heart_assign_thresholds: no assignment meets the budget */
 };
 
 #define HEART_FORCE_REFRESH 1u /* every head refreshes this step (decision overridden)  */
@@ -240,6 +241,28 @@ size_t heart_band_error_workspace_bytes(int32_t C, int32_t T, int32_t H, int32_t
 int heart_band_error(const float *y_sparse, const float *y_dense, int32_t C, int32_t T, int32_t H, int32_t W,
                      const double *weights /* host [4] */, double eps, double *out, void *workspace,
                      heart_stream_t stream);
+
+/* Threshold assignment of the offline calibration -- the one-choice-per-head assignment problem of the
+ * section "Error-guided Budgeted Calibration" (the last step of Algorithm 2; appendix "Optimization
+ * and budget": three candidate thresholds 0.85 / 0.90 / 0.95 per head):
+ *     minimise   sum_i E[i][k_i]
+ *     subject to one candidate k_i per head i  and  (1/M) sum_i S[i][k_i] >= S_min.
+ * An offline problem on M * K numbers: it runs on the HOST (every pointer here is a host pointer, no
+ * GPU is touched) as an exact multiple-choice-knapsack search.
+ *   E, S: [n_heads, n_candidates] row-major fp64, the measured error and realised sparsity of each
+ *   candidate of each head (the heads of all layers flattened); finite values.
+ *   choice_out [n_heads]: the chosen candidate index per head.  objective_out, mean_sparsity_out
+ *   (optional): the plain left-to-right sums of the chosen entries (the second divided by n_heads) --
+ *   the same arithmetic that decides feasibility.  proved_optimal_out (optional): 1 when the search
+ *   ran to the end (always, short of pathological tables with tens of millions of undominated
+ *   partial sums), 0 when it stopped early and returns the best assignment found.
+ * Among assignments of exactly equal objective any one may be returned.
+ * Returns HEART_ERR_INFEASIBLE (outputs untouched) when even the sparsest candidate of every head
+ * misses the budget. */
+int heart_assign_thresholds(const double *E /* host */, const double *S /* host */, int32_t n_heads,
+                            int32_t n_candidates, double S_min, int32_t *choice_out /* host */,
+                            double *objective_out /* host */, double *mean_sparsity_out /* host */,
+                            int32_t *proved_optimal_out /* host */);
 
 /* Synchronises `stream`, reads the workspace status word into *code_out (host) and clears it.
  * The only call that blocks. */

@@ -27,6 +27,10 @@
  *                                              uniform-row closed form, limits)
  *   masked attention ......................... pinned (dense brute force, library
  *                                              attention, closed forms)
+ *   threshold assignment under a budget ...... pinned (an independent MILP
+ *                                              solver, forced / unconstrained /
+ *                                              infeasible cases, a hand-worked
+ *                                              two-head table, monotonicity)
  *   fidelity of the block-importance estimator to the paper's third-party
  *   backbones (antidiagonal scoring / k-means) ........ parity unpinned: the
  *   paper does not define them; the estimator here is mean-pooled Q.K^T.
@@ -489,4 +493,51 @@ void oracle_mask_iou(const uint32_t *mask_a, const uint32_t *mask_b, int R, int 
       counts[2 * r + 1] = uni;
     }
   }
+}
+
+/* ---------------------------------------------------------------------------
+ * Threshold assignment of the offline calibration (section "Error-guided
+ * Budgeted Calibration", the one-choice-per-head assignment problem; last step
+ * of Algorithm 2):
+ *     minimise   sum_i E[i][k_i]
+ *     subject to one candidate k_i per head i,  (1/M) sum_i S[i][k_i] >= S_min.
+ * E, S: [M][K] measured error and realised sparsity of candidate k of head i
+ * (heads of all layers flattened, M = L*H).  Written out as the definition:
+ * every one of the K^M assignments is visited in lexicographic order (the last
+ * head varies fastest), both sums are plain left-to-right loops over the heads,
+ * and an assignment replaces the best one only if its objective is strictly
+ * smaller -- so among exactly equal objectives the lexicographically first
+ * wins.  For M up to about a dozen heads.
+ * Returns 1 and fills choice[M], *objective, *mean_sparsity; returns 0 when no
+ * assignment meets the budget (outputs untouched).
+ * ------------------------------------------------------------------------ */
+int oracle_assign_thresholds(const double *E, const double *S, int M, int K, double S_min, int32_t *choice,
+                             double *objective, double *mean_sparsity) {
+  if (M <= 0 || K <= 0) return 0;
+  int *k = (int *)calloc((size_t)M, sizeof(int));
+  int found = 0;
+  double best = 0.0, best_s = 0.0;
+  for (;;) {
+    double e = 0.0, s = 0.0;
+    for (int i = 0; i < M; ++i) {
+      e += E[(size_t)i * K + k[i]];
+      s += S[(size_t)i * K + k[i]];
+    }
+    s /= (double)M;
+    if (s >= S_min && (!found || e < best)) {
+      found = 1;
+      best = e;
+      best_s = s;
+      for (int i = 0; i < M; ++i) choice[i] = k[i];
+    }
+    int i = M - 1;
+    while (i >= 0 && ++k[i] == K) k[i--] = 0;
+    if (i < 0) break;
+  }
+  free(k);
+  if (found) {
+    if (objective) *objective = best;
+    if (mean_sparsity) *mean_sparsity = best_s;
+  }
+  return found;
 }

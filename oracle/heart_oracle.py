@@ -1,9 +1,11 @@
 """ctypes front end of the CPU oracle (oracle/heart_oracle.c).
 
 TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
-benchmark's CPU-baseline leg.  Holds no arithmetic of its own -- every number
-comes from the C functions; this file only builds the shared object with gcc,
-marshals numpy arrays and allocates outputs.
+benchmark's CPU-baseline leg.  For the layer-step path this file holds no
+arithmetic of its own -- every number comes from the C functions; it only builds
+the shared object with gcc, marshals numpy arrays and allocates outputs.  The one
+exception is at the end: band_error (the offline calibration's four-band
+spectral error) is written here, in numpy, straight from its definition.
 
 bf16 tensors are passed as numpy uint16 arrays holding the raw bf16 bits,
 contiguous [R, N, D] (R = batch * heads).
@@ -228,6 +230,20 @@ def mask_iou(mask_a, mask_b, nb):
     counts = np.empty((R, 2), np.int64)
     lib().oracle_mask_iou(_p(mask_a), _p(mask_b), R, int(nb), _p(iou), _p(counts))
     return iou, counts
+
+
+def assign_thresholds(E, S, S_min):
+    """One-choice-per-head assignment under a sparsity budget by exhaustive enumeration.
+    E, S: [M, K].  Returns (choice[M] int32, objective, mean sparsity) or None when infeasible."""
+    E = np.ascontiguousarray(E, np.float64)
+    S = np.ascontiguousarray(S, np.float64)
+    M, K = E.shape
+    assert S.shape == (M, K) and K ** M <= 20_000_000, "exhaustive: keep K^M small"
+    choice = np.empty(M, np.int32)
+    obj, ms = C.c_double(0), C.c_double(0)
+    lib().oracle_assign_thresholds.restype = C.c_int
+    ok = lib().oracle_assign_thresholds(_p(E), _p(S), M, K, C.c_double(S_min), _p(choice), C.byref(obj), C.byref(ms))
+    return (choice, obj.value, ms.value) if ok else None
 
 
 # ---------------------------------------------------------------------------

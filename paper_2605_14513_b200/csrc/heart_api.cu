@@ -390,6 +390,7 @@ const char *heart_strerror(int code) {
     case HEART_ERR_UNSUPPORTED: return "unsupported shape (head_dim must be 128, block 64 or 128, at most 1024 blocks)";
     case HEART_ERR_CUDA: return g_errbuf[0] ? g_errbuf : "CUDA error";
     case HEART_ERR_TOO_LARGE: return "shape needs more scratch than the built-in HEART_STATIC_SCRATCH_BYTES array holds";
+    case HEART_ERR_INFEASIBLE: return "no assignment of one candidate per head meets the sparsity budget";
     case HEART_ERR_DEVICE_CHECK: return "device-side check failed (index-list entry out of range or a bounded wait ran out)";
     default: return "unknown code";
   }

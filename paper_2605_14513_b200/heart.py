@@ -14,7 +14,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.environ.get("HEART_LIB") or os.path.join(_HERE, "libheart.so")
 
-OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TOO_LARGE = 0, 1, 2, 3, 4, 5
+OK, ERR_INVALID, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_CHECK, ERR_TOO_LARGE, ERR_INFEASIBLE = 0, 1, 2, 3, 4, 5, 6
 STATIC_SCRATCH_BYTES = 16 << 20
 FORCE_REFRESH, FORCE_DENSE, BLOCK_MEANS_VALID, ESTIMATOR_ANTIDIAG = 1, 2, 4, 8
 MAX_BLOCKS = 1024
@@ -25,6 +25,7 @@ SYMBOLS = (
     "heart_block_sparse_attn", "heart_step", "heart_step_host", "heart_get_status", "heart_strerror",
     "heart_last_launch_count", "heart_drift_static", "heart_full_token_drift", "heart_mask_iou",
     "heart_band_error_workspace_bytes", "heart_band_error", "heart_drift_workspace_bytes",
+    "heart_assign_thresholds",
 )
 
 
@@ -83,6 +84,9 @@ def lib():
         l.heart_band_error_workspace_bytes.restype = C.c_size_t
         l.heart_band_error.argtypes = [vp, vp] + [C.c_int32] * 4 + [C.POINTER(C.c_double), C.c_double, vp, vp, vp]
         l.heart_band_error.restype = C.c_int
+        l.heart_assign_thresholds.argtypes = [vp, vp, C.c_int32, C.c_int32, C.c_double, vp, C.POINTER(C.c_double),
+                                              C.POINTER(C.c_double), C.POINTER(C.c_int32)]
+        l.heart_assign_thresholds.restype = C.c_int
         for fn in ("heart_state_reset", "heart_drift", "heart_predict_mask", "heart_block_sparse_attn",
                    "heart_step", "heart_step_host", "heart_get_status"):
             getattr(l, fn).restype = C.c_int
@@ -243,6 +247,27 @@ def heart_band_error(y_sparse, y_dense, weights=(1.0, 0.5, 0.01, 0.01), eps=1e-1
     _check(lib().heart_band_error(_ptr(y_sparse), _ptr(y_dense), Cc, T, H, W, w, float(eps), _ptr(out), _ptr(ws),
                                   _stream()))
     return out
+
+
+def heart_assign_thresholds(E, S, S_min):
+    """One threshold candidate per head under a mean-sparsity budget (host-side, exact).
+    E, S: [n_heads, n_candidates] float64 numpy arrays.  Returns (choice int32 [n_heads], objective,
+    mean sparsity, proved_optimal) or None when no assignment meets the budget."""
+    import numpy as np
+
+    E = np.ascontiguousarray(E, np.float64)
+    S = np.ascontiguousarray(S, np.float64)
+    M, K = E.shape
+    assert S.shape == (M, K)
+    choice = np.empty(M, np.int32)
+    obj, ms, proved = C.c_double(0), C.c_double(0), C.c_int32(0)
+    rc = lib().heart_assign_thresholds(E.ctypes.data_as(C.c_void_p), S.ctypes.data_as(C.c_void_p), M, K,
+                                       float(S_min), choice.ctypes.data_as(C.c_void_p), C.byref(obj), C.byref(ms),
+                                       C.byref(proved))
+    if rc == ERR_INFEASIBLE:
+        return None
+    _check(rc)
+    return choice, obj.value, ms.value, bool(proved.value)
 
 
 def heart_get_status(ws) -> int:
