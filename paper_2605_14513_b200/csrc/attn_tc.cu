@@ -74,6 +74,7 @@ struct AttnBars {
   uint64_t qk_done[kStages];                  // S_h complete: softmax may read it, K stage is free
   uint64_t pv_done[kStages];                  // P_h V_h complete: V stage and S/P buffer are free
   uint64_t p_full[kStages];                   // P_h written (one arrival per warp of the stream)
+  uint64_t drain[2];                          // abort path: the issuers' products in flight have landed
   uint32_t tmem_base;
   int chunk_cnt[32];  // flagged key blocks per 32-block chunk (set-up)
   int n_union;
@@ -93,6 +94,7 @@ struct AttnParams {
   const int32_t *order;   // the last n_sorted CTAs take their tile from this table (longest lists first)
   int n_sorted;
   float scale_log2;
+  int test_skip_v;  // test-hook builds only: CTA 0 leaves out the V copy of its second key step
 };
 
 // Clock-stamp trace (compile with -DHEART_TRACE; the caller's lse buffer must then have one extra
@@ -181,6 +183,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
       mbar_init(&bars->pv_done[i], 1);
       mbar_init(&bars->p_full[i], 4);  // one arrival per softmax warp
     }
+    mbar_init(&bars->drain[0], 1);
+    mbar_init(&bars->drain[1], 1);
     bars->abort = 0;
     bars->bad = 0;
     bars->n_union = 0;
@@ -340,6 +344,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
       for (int h = 0; h < NH; ++h) {
         const int s = h % kStages, ph = (h / kStages) & 1;
         if (h >= kStages && !mbar_wait_relaxed(&bars->pv_done[s], ph ^ 1, abort)) break;
+#ifdef HEART_TEST_HOOKS
+        // Test-only library: one V tile is never requested (neither the byte count nor the copy), so the
+        // waits that depend on it run out and the abort path below is taken.
+        if (p.test_skip_v && blockIdx.x == 0 && h == 1) continue;
+#endif
         const int key0 = key0_of(h);
         unsigned char *dst = Vs + s * L::KV_BYTES;
         mbar_expect_tx(&bars->v_full[s], L::KV_BYTES);
@@ -422,6 +431,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
           __syncwarp();
           HEART_TR(h, 9);
         }
+      }
+      if (*abort) {
+        // Tensor memory must not be released under a product in flight: a commit arrives once
+        // everything this lane has issued is complete; the wait for it is bounded like the others.
+        uint64_t *bar = &bars->drain[warp == kWarpQK ? 0 : 1];
+        if (leader) tc_commit(bar);
+        __syncwarp();
+        settle(bar, 0);
       }
     }
   } else {
@@ -712,6 +729,10 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
   prm.R_all = g.R;
   prm.scale_log2 = (float)(g.scale * 1.4426950408889634);
   prm.order = order;
+  prm.test_skip_v = 0;
+#ifdef HEART_TEST_HOOKS
+  prm.test_skip_v = (g.flags & 0x80000000u) ? 1 : 0;
+#endif
   prm.n_sorted = 0;
   if (!dense && order != nullptr) {
     const int rows = g.B * hcount, nlast = rows < 2 ? rows : 2, n = nlast * prm.n_ctas_per_head;

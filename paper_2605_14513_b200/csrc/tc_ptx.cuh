@@ -44,7 +44,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity, ui
 
 // Bounded wait: gives up after `kWaitLimitCycles` SM clocks or as soon as another thread of the
 // CTA has raised *abort.  Returns false in both cases (and raises *abort on a time-out).
-constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at 1.9 GHz; a real wait is microseconds
+#ifndef HEART_WAIT_LIMIT_CYCLES
+#define HEART_WAIT_LIMIT_CYCLES 4000000000LL  // ~2 s at 1.9 GHz; a real wait is microseconds
+#endif
+constexpr long long kWaitLimitCycles = HEART_WAIT_LIMIT_CYCLES;
 __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity) {  // never blocks
   uint32_t ok;
   asm volatile(

@@ -55,10 +55,18 @@ def lib():
     """The loaded libheart.so (raises if it is missing: build it with build.py)."""
     global _lib
     if _lib is None:
-        if not os.path.exists(_LIB_PATH):
-            raise ImportError(f"{_LIB_PATH} not found: run `python -m paper_2605_14513_b200.build` "
+        _lib = load(_LIB_PATH)
+    return _lib
+
+
+def load(path):
+    """Loads a build of the library and declares its signatures (the tests use this for the
+    test-hook build; everything else goes through lib())."""
+    if True:
+        if not os.path.exists(path):
+            raise ImportError(f"{path} not found: run `python -m paper_2605_14513_b200.build` "
                               "(or __graft_entry__.build()) -- there is no fallback path")
-        l = C.CDLL(_LIB_PATH)
+        l = C.CDLL(path)
         l.heart_workspace_bytes.restype = C.c_size_t
         l.heart_workspace_bytes.argtypes = [C.POINTER(Config)]
         l.heart_drift_workspace_bytes.restype = C.c_size_t
@@ -90,8 +98,7 @@ def lib():
         for fn in ("heart_state_reset", "heart_drift", "heart_predict_mask", "heart_block_sparse_attn",
                    "heart_step", "heart_step_host", "heart_get_status"):
             getattr(l, fn).restype = C.c_int
-        _lib = l
-    return _lib
+    return l
 
 
 def _ptr(t):

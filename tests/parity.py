@@ -76,6 +76,17 @@ def check_masks(gpu_state, ref_state, heads, tau, probs_row_fn):
     return exempt
 
 
+def attention_abs_bound(O_ref):
+    """Element-wise absolute bound on |O_gpu - O_ref|.  The output is stored as bf16 (8 significant
+    bits), so rounding alone costs up to half a unit in the last place: 2^(e-8) for |O| in
+    [2^e, 2^(e+1)), i.e. 0.0078 on [2, 4) and 0.0156 on [4, 8).  Below 4 the flat 2e-2 of the
+    acceptance bar covers that rounding plus the ~5e-3 the fp32 accumulation of bf16-rounded weights
+    contributes; from 4 up the bound is that same 5e-3 on top of the half-ulp of the value itself."""
+    mag = np.abs(np.asarray(O_ref, np.float64))
+    half_ulp = np.exp2(np.floor(np.log2(np.maximum(mag, 1e-30))) - 8.0)
+    return np.where(mag < 4.0, ATTN_MAX_ABS, half_ulp + 5e-3)
+
+
 def check_attention(O_gpu, O_ref, valid=None):
     """O_gpu: float array widened from bf16; O_ref: fp64 oracle; both [..., D]."""
     a = np.asarray(O_gpu, np.float64)
@@ -83,9 +94,11 @@ def check_attention(O_gpu, O_ref, valid=None):
     if valid is not None:
         a, b = a[valid], b[valid]
     assert np.isfinite(a).all()
-    max_abs = np.abs(a - b).max()
+    err = np.abs(a - b)
+    max_abs = err.max()
     rel_l2 = math.sqrt(((a - b) ** 2).sum() / max((b ** 2).sum(), 1e-300))
-    assert max_abs <= ATTN_MAX_ABS, f"max-abs {max_abs}"
+    over = err > attention_abs_bound(b)
+    assert not over.any(), f"max-abs {max_abs} (worst excess {(err - attention_abs_bound(b)).max()})"
     assert rel_l2 <= ATTN_REL_L2, f"rel-L2 {rel_l2}"
     return max_abs, rel_l2
 
@@ -138,9 +151,13 @@ class Pair:
 
 
 def sample_rows(rs, R, nb, kv_cnt, n):
-    """(r, I) sample: row 0, the ragged last block, the densest and the sparsest row, then random."""
+    """(r, I) sample: row 0, the ragged last block, the densest and the sparsest row; two adjacent query
+    blocks (the two halves of one 128-row tile at block 64) of the first head, whose tiles run in index
+    order, and of the last head, whose tiles the attention launch orders longest-first; then random."""
     flat = kv_cnt.reshape(-1)
     picks = {(0, 0), (R - 1, nb - 1), divmod(int(flat.argmax()), nb), divmod(int(flat.argmin()), nb)}
+    if nb >= 4:
+        picks |= {(0, 0), (0, 1), (R - 1, 2), (R - 1, 3)}
     while len(picks) < n:
         picks.add((int(rs.randint(R)), int(rs.randint(nb))))
     picks = sorted(picks)
