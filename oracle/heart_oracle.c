@@ -31,9 +31,15 @@
  *                                              solver, forced / unconstrained /
  *                                              infeasible cases, a hand-worked
  *                                              two-head table, monotonicity)
- *   fidelity of the block-importance estimator to the paper's third-party
+ *   strided antidiagonal estimator ........... pinned as defined here (token-level
+ *                                              brute force, stride 1 = dense softmax
+ *                                              block sums, single-pair and shift
+ *                                              closed forms); its fidelity to the
+ *                                              paper's backbone is PARITY UNPINNED
+ *   fidelity of the block-importance estimators to the paper's third-party
  *   backbones (antidiagonal scoring / k-means) ........ parity unpinned: the
- *   paper does not define them; the estimator here is mean-pooled Q.K^T.
+ *   paper does not define them; the default estimator here is mean-pooled
+ *   Q.K^T, the alternative one is the strided antidiagonal sum defined below.
  */
 #include <math.h>
 #include <stdint.h>
@@ -540,4 +546,92 @@ int oracle_assign_thresholds(const double *E, const double *S, int M, int K, dou
     if (mean_sparsity) *mean_sparsity = best_s;
   }
   return found;
+}
+
+/* ---------------------------------------------------------------------------
+ * Strided antidiagonal block-importance estimator -- the estimator family the
+ * paper's main backbone uses (appendix "XAttention and SVG2 Configurations":
+ * anti-diagonal scoring with stride 16 on 128-token blocks; the paper gives
+ * only those two numbers, so the definition below is this build's own, and its
+ * fidelity to that backbone is PARITY UNPINNED):
+ *   the sequence is cut into groups of s consecutive tokens; only the
+ *   Ns = floor(N / s) full groups are sampled (trailing tokens are not seen);
+ *   S'(a, c) = (scale / s) * sum_{t<s} <q_{a s + t}, k_{c s + s-1-t}>
+ *            = the mean of the s token-level logits on the antidiagonal of the
+ *              s x s tile (group a, group c);
+ *   P'(a, .) = softmax over the Ns groups c (two-pass);
+ *   importance of block pair (I, J) = sum of P'(a, c) over the groups a inside
+ *   query block I and the groups c inside key block J, divided by the number of
+ *   groups in I, so every row sums to 1.  A query block with no full group has
+ *   uniform importance 1/nb; a key block with no full group has importance 0.
+ * (s must divide b.)  P receives the nb importances of query block I of head r.
+ * ------------------------------------------------------------------------ */
+void oracle_antidiag_probs_row(const uint16_t *Q, const uint16_t *K, int N, int D, int b, int s,
+                               double scale, int r, int I, double *P) {
+  int nb = (N + b - 1) / b, Ns = N / s, g = b / s;
+  if (!(scale > 0.0)) scale = 1.0 / sqrt((double)D);
+  const uint16_t *Qr = Q + (size_t)r * N * D, *Kr = K + (size_t)r * N * D;
+  int a0 = I * g, a1 = a0 + g < Ns ? a0 + g : Ns;
+  if (a1 <= a0) {
+    for (int J = 0; J < nb; ++J) P[J] = 1.0 / (double)nb;
+    return;
+  }
+  for (int J = 0; J < nb; ++J) P[J] = 0.0;
+  double *row = (double *)malloc(sizeof(double) * (size_t)Ns);
+  for (int a = a0; a < a1; ++a) {
+    for (int c = 0; c < Ns; ++c) {
+      double acc = 0.0;
+      for (int t = 0; t < s; ++t) {
+        const uint16_t *q = Qr + (size_t)(a * s + t) * D, *k = Kr + (size_t)(c * s + s - 1 - t) * D;
+        for (int d = 0; d < D; ++d) acc += bf16_to_double(q[d]) * bf16_to_double(k[d]);
+      }
+      row[c] = acc * (scale / (double)s);
+    }
+    double mx = row[0];
+    for (int c = 1; c < Ns; ++c) mx = row[c] > mx ? row[c] : mx;
+    double z = 0.0;
+    for (int c = 0; c < Ns; ++c) {
+      row[c] = exp(row[c] - mx);
+      z += row[c];
+    }
+    for (int c = 0; c < Ns; ++c) P[c / g] += row[c] / z;
+  }
+  for (int J = 0; J < nb; ++J) P[J] /= (double)(a1 - a0);
+  free(row);
+}
+
+/* Mask prediction with that estimator in place of the pooled one: the importances of every query
+ * block go through the same top-p rule (oracle_top_p) with the head's tau.  Heads with
+ * refresh[r] == 0 are left untouched; refresh == NULL means all heads. */
+void oracle_predict_mask_antidiag(const uint16_t *Q, const uint16_t *K, int R, int N, int D, int b, int s,
+                                  double scale, const double *tau, const uint8_t *refresh, uint32_t flags,
+                                  uint32_t *mask_bits, int32_t *kv_idx, int32_t *kv_cnt, int idx_stride) {
+  int nb = (N + b - 1) / b;
+  int W = (nb + 31) / 32;
+  for (int r = 0; r < R; ++r) {
+    if (refresh && !refresh[r]) continue;
+#pragma omp parallel
+    {
+      double *P = (double *)malloc(sizeof(double) * (size_t)nb);
+      uint8_t *keep = (uint8_t *)malloc((size_t)nb);
+#pragma omp for schedule(dynamic, 1)
+      for (int I = 0; I < nb; ++I) {
+        oracle_antidiag_probs_row(Q, K, N, D, b, s, scale, r, I, P);
+        double t = (flags & ORACLE_FORCE_DENSE) ? 1.0 : tau[r];
+        oracle_top_p(P, nb, t, keep, NULL, NULL);
+        uint32_t *bits = mask_bits + ((size_t)r * nb + I) * W;
+        int32_t *idx = kv_idx + ((size_t)r * nb + I) * idx_stride;
+        memset(bits, 0, sizeof(uint32_t) * (size_t)W);
+        int c = 0;
+        for (int J = 0; J < nb; ++J)
+          if (keep[J]) {
+            bits[J >> 5] |= 1u << (J & 31);
+            idx[c++] = J;
+          }
+        kv_cnt[(size_t)r * nb + I] = c;
+      }
+      free(P);
+      free(keep);
+    }
+  }
 }

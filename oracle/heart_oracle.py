@@ -157,6 +157,31 @@ def predict_mask(Q, K, b, tau, st: State, refresh=None, scale=0.0, flags=0):
                               st.idx_stride)
 
 
+ANTIDIAG_STRIDE = 16
+
+
+def antidiag_probs_row(Q, K, b, r, I, s=ANTIDIAG_STRIDE, scale=0.0):
+    """Block importances of query block I of head r under the strided antidiagonal estimator."""
+    Q, K = _u16(Q), _u16(K)
+    R, N, D = Q.shape
+    assert b % s == 0
+    P = np.empty(n_blocks(N, b), np.float64)
+    lib().oracle_antidiag_probs_row(_p(Q), _p(K), N, D, b, int(s), C.c_double(scale), int(r), int(I), _p(P))
+    return P
+
+
+def predict_mask_antidiag(Q, K, b, tau, st: State, refresh=None, s=ANTIDIAG_STRIDE, scale=0.0, flags=0):
+    Q, K = _u16(Q), _u16(K)
+    R, N, D = Q.shape
+    assert b % s == 0
+    tau = np.ascontiguousarray(tau, np.float64)
+    if refresh is not None:
+        refresh = np.ascontiguousarray(refresh, np.uint8)
+    lib().oracle_predict_mask_antidiag(_p(Q), _p(K), R, N, D, b, int(s), C.c_double(scale), _p(tau), _p(refresh),
+                                       C.c_uint32(flags), _p(st.mask_bits), _p(st.kv_idx), _p(st.kv_cnt),
+                                       st.idx_stride)
+
+
 def probs_row(Q, K, b, r, I, scale=0.0):
     Q, K = _u16(Q), _u16(K)
     R, N, D = Q.shape
