@@ -63,7 +63,9 @@ enum {
 #define HEART_BLOCK_MEANS_VALID 4u /* heart_predict_mask only: the workspace already holds */
                                /* the block means of these Q, K (see that call)          */
 #define HEART_ESTIMATOR_ANTIDIAG 8u /* mask prediction ranks blocks with the strided       */
-                               /* antidiagonal estimator instead of mean pooling         */
+                               /* antidiagonal estimator instead of mean pooling (see    */
+                               /* heart_predict_mask); needs a larger workspace          */
+#define HEART_ANTIDIAG_STRIDE 16   /* tokens per sampled group of that estimator          */
 
 #define HEART_MAX_BLOCKS 1024  /* largest supported n_b */
 
@@ -90,7 +92,8 @@ typedef struct {
 
 /* Bytes of scratch every compute call needs (block means, token means, flags, status
  * word, and the pooled scores of the mask predictor: 8 * R * n_b * roundup(n_b, 32) bytes,
- * by far the largest part).  Host-only; returns 0 for an invalid or unsupported config.
+ * by far the largest part; with HEART_ESTIMATOR_ANTIDIAG in cfg->flags another
+ * 8 * R * floor(N / 16) * n_b bytes).  Host-only; returns 0 for an invalid or unsupported config.
  * The caller allocates it once (256-byte aligned) and zero-fills it before first use. */
 size_t heart_workspace_bytes(const heart_config *cfg /* host */);
 
@@ -123,7 +126,18 @@ int heart_drift(const heart_config *cfg, const void *Q, const void *K, const dou
  *   kept: tau[r] <= 0 keeps exactly the largest block (the lowest index among equals).
  * Writes mask_bits, kv_idx (ascending), kv_cnt of those heads; other heads are untouched.
  * tau [R] fp64.
- * The call first repeats heart_drift's pass over Q and K for the block means.  A caller that has just
+ * With HEART_ESTIMATOR_ANTIDIAG in cfg->flags the importances come from the strided antidiagonal
+ * estimator instead (the estimator family of the paper's main sparse-attention backbone, appendix
+ * "XAttention and SVG2 Configurations": anti-diagonal scoring with stride 16; the paper states the
+ * stride and the block size only, so the definition is this library's):
+ *   tokens are taken in groups of s = HEART_ANTIDIAG_STRIDE; only the floor(N / s) full groups are
+ *   sampled;  S'(a, c) = (scale / s) * sum_{t<s} <q_{a s + t}, k_{c s + s-1-t}>;  P'(a, .) = softmax over
+ *   the groups c;  P[r,I,J] = sum of P'(a, c) over the groups of blocks I and J / groups in I;
+ *   a query block without a full group gets uniform P, a key block without one gets P = 0;
+ *   then the same selection rule.  The contraction runs in bf16 with fp32 accumulation on the tensor
+ *   cores, the exponentials in fp32, the block sums and the selection in fp64.  The workspace must
+ *   have been sized with the flag set.  heart_step and heart_step_host honour the flag too.
+ * (Pooled estimator:) the call first repeats heart_drift's pass over Q and K for the block means.  A caller that has just
  * run heart_drift (or heart_predict_mask) on the same Q and K pointers, the same cfg shape and the
  * same workspace, with no heart_full_token_drift and no change of the tensors' contents in between,
  * sets HEART_BLOCK_MEANS_VALID in cfg->flags: the pass is skipped and the means in the workspace are

@@ -46,6 +46,8 @@ struct Workspace {
   double *drift;      // [R]
   int32_t *order;     // [2048] tile order of the last two heads of an attention launch
   double *scores;     // [R][nb][pitch] pooled scores of the refreshed heads, pitch = nb rounded up to 32
+  void *pairs;        // strided antidiagonal estimator only (HEART_ESTIMATOR_ANTIDIAG in the flags):
+                      // float2 [R][N/16][nb], a (max, sum) pair per (query group, key block)
   size_t bytes_drift;  // what heart_drift alone touches (everything above `scores`)
   size_t bytes;
 };
@@ -75,6 +77,9 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   w.bytes_drift = off;
   w.scores = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * (size_t)g.R * g.nb * (size_t)(((g.nb + 31) / 32) * 32));
+  w.pairs = p + off;
+  if (g.flags & HEART_ESTIMATOR_ANTIDIAG)
+    off += align256(8 * (size_t)g.R * (size_t)(g.N / HEART_ANTIDIAG_STRIDE) * (size_t)g.nb);
   w.bytes = off;
   return w;
 }
@@ -121,6 +126,14 @@ cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta
 cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
                                 const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches,
                                 unsigned long long expect_sig = 0);
+// The two halves of it: pooled scores into w.scores, then the top-p rows over w.scores.
+cudaError_t launch_pooled_scores(const Geom &g, const Workspace &w, const uint8_t *refresh, cudaStream_t s,
+                                 int *launches, unsigned long long expect_sig);
+cudaError_t launch_top_p(const Geom &g, const Workspace &w, const double *tau, const uint8_t *refresh,
+                         heart_state st, cudaStream_t s, int *launches, unsigned long long expect_sig);
+// Strided antidiagonal estimator: log block importances of the refreshed heads into w.scores.
+cudaError_t launch_antidiag_scores(const Geom &g, const Workspace &w, const void *Q, const void *K,
+                                   const uint8_t *refresh, cudaStream_t s, int *launches);
 // h0/hcount select the heads [h0, h0 + hcount) of every batch entry (hcount <= 0: all heads).
 cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const void *V,
                              const int32_t *kv_idx, const int32_t *kv_cnt, bool dense, void *O,

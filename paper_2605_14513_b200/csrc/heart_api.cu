@@ -66,6 +66,17 @@ bool state_ok(const heart_state *st) {
   return st && st->anchor_q && st->anchor_k && st->has_anchor && st->mask_bits && st->kv_idx && st->kv_cnt;
 }
 
+// Mask prediction inside a layer-step (the refresh flags are the ones the decision kernel just wrote).
+cudaError_t predict_for_step(const Geom &g, const Workspace &w, const void *Q, const void *K, const double *tau,
+                             heart_state st, cudaStream_t s) {
+  if (g.flags & HEART_ESTIMATOR_ANTIDIAG) {
+    cudaError_t e = launch_antidiag_scores(g, w, Q, K, w.refresh, s, &g_launches);
+    if (e != cudaSuccess) return e;
+    return launch_top_p(g, w, tau, w.refresh, st, s, &g_launches, 0);
+  }
+  return launch_predict_mask(g, w, tau, w.refresh, st, s, &g_launches);
+}
+
 __global__ void fill_dense_outputs_kernel(int R, double *drift_out, uint8_t *refresh_out, uint8_t *refresh_ws) {
   const int r = blockIdx.x * blockDim.x + threadIdx.x;
   if (r < R) {
@@ -134,6 +145,14 @@ int heart_predict_mask(const heart_config *cfg, const void *Q, const void *K, co
   g_launches = 0;
   cudaError_t e;
   unsigned long long expect_sig = 0;
+  if (g.flags & HEART_ESTIMATOR_ANTIDIAG) {
+    // this estimator works on the tokens themselves: no block means needed
+    e = launch_antidiag_scores(g, w, Q, K, refresh, s, &g_launches);
+    if (e != cudaSuccess) return cuda_fail(e, "antidiag_scores");
+    e = launch_top_p(g, w, tau, refresh, *st, s, &g_launches, 0);
+    if (e != cudaSuccess) return cuda_fail(e, "top_p");
+    return HEART_OK;
+  }
   if (g.flags & HEART_BLOCK_MEANS_VALID) {
     // the caller vouches that a heart_drift (or heart_predict_mask) on these very tensors left the block
     // means in this workspace: no second pass over Q and K; the kernels verify the workspace's signature
@@ -193,7 +212,7 @@ int heart_step(const heart_config *cfg, const void *Q, const void *K, const void
   if (e != cudaSuccess) return cuda_fail(e, "block_sums");
   e = launch_decide(g, w, delta, *st, drift_out, refresh_out, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "decide");
-  e = launch_predict_mask(g, w, tau, w.refresh, *st, s, &g_launches);
+  e = predict_for_step(g, w, Q, K, tau, *st, s);
   if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
   e = launch_attention(g, Q, K, V, st->kv_idx, st->kv_cnt, false, O, lse, w.status, w.order, s, &g_launches);
   if (e != cudaSuccess) return cuda_fail(e, "attention");
@@ -278,7 +297,7 @@ int heart_step_host(const heart_config *cfg, const void *Q_host, const void *K_h
     if (e != cudaSuccess) return cuda_fail(e, "block_sums");
     e = launch_decide(g, w, delta, *st, w.drift, nullptr, s, &g_launches);
     if (e != cudaSuccess) return cuda_fail(e, "decide");
-    e = launch_predict_mask(g, w, tau, w.refresh, *st, s, &g_launches);
+    e = predict_for_step(g, w, Q_dev, K_dev, tau, *st, s);
     if (e != cudaSuccess) return cuda_fail(e, "predict_mask");
   }
   const int groups = g.H < kHostGroups ? g.H : kHostGroups;

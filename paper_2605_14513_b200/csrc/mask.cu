@@ -386,22 +386,34 @@ static cudaError_t launch_nj(const Geom &g, const Workspace &w, const double *ta
                     expect_sig);
 }
 
-cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
-                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches,
-                                unsigned long long expect_sig) {
-  *launches += 2;
+cudaError_t launch_pooled_scores(const Geom &g, const Workspace &w, const uint8_t *refresh, cudaStream_t s,
+                                 int *launches, unsigned long long expect_sig) {
+  ++*launches;
   const int nj = (g.nb + 31) / 32, pitch = nj * 32;
   const size_t smem = sizeof(double) * 2 * (SI + SJ) * KLD;
   cudaError_t e = cudaFuncSetAttribute(pooled_scores_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   dim3 grid((g.nb + SJ - 1) / SJ, (g.nb + SI - 1) / SI, g.R);
-  e = launch_pdl(pooled_scores_kernel, grid, dim3(256), smem, s, (const double *)w.bmean, g.R, g.nb, pitch, g.scale,
-                 refresh, w.scores, w.status, expect_sig);
-  if (e != cudaSuccess) return e;
+  return launch_pdl(pooled_scores_kernel, grid, dim3(256), smem, s, (const double *)w.bmean, g.R, g.nb, pitch, g.scale,
+                    refresh, w.scores, w.status, expect_sig);
+}
+
+cudaError_t launch_top_p(const Geom &g, const Workspace &w, const double *tau, const uint8_t *refresh,
+                         heart_state st, cudaStream_t s, int *launches, unsigned long long expect_sig) {
+  ++*launches;
+  const int nj = (g.nb + 31) / 32, pitch = nj * 32;
   if (nj <= 8) return launch_nj<8>(g, w, tau, refresh, st, pitch, s, expect_sig);
   if (nj <= 16) return launch_nj<16>(g, w, tau, refresh, st, pitch, s, expect_sig);
   if (nj <= 24) return launch_nj<24>(g, w, tau, refresh, st, pitch, s, expect_sig);
   return launch_nj<32>(g, w, tau, refresh, st, pitch, s, expect_sig);
+}
+
+cudaError_t launch_predict_mask(const Geom &g, const Workspace &w, const double *tau,
+                                const uint8_t *refresh, heart_state st, cudaStream_t s, int *launches,
+                                unsigned long long expect_sig) {
+  cudaError_t e = launch_pooled_scores(g, w, refresh, s, launches, expect_sig);
+  if (e != cudaSuccess) return e;
+  return launch_top_p(g, w, tau, refresh, st, s, launches, expect_sig);
 }
 
 }  // namespace heart
