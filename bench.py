@@ -327,6 +327,36 @@ def measure(torch, heart, inputs, replicas, wl, K, W, dev, pk, rank, sampler_uui
         torch.cuda.synchronize()
         dense_ms = a.elapsed_time(b_) / 3
 
+    # ---- mask prediction with every head refreshing, both estimators, on the first timed step's tensors:
+    # the pooled one (the block means are in the workspace: heart_drift has just run) and the strided
+    # antidiagonal one (a bf16 contraction per head on the tensor cores, in a workspace of its own size)
+    Q, Kt, V = steps_in[W]
+    st_m = heart.State(cfg, dev)
+
+    def timed(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b_.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b_) / reps
+
+    heart.heart_drift(cfg, Q, Kt, delta, st_m, ws)
+    ms_mask_pooled_all = timed(lambda: heart.heart_predict_mask(cfg, Q, Kt, tau, st_m, ws, means_valid=True), 5)
+    dens_pooled = float(st_m.kv_cnt.to(torch.float64).mean()) / wl.n_blocks
+    cfg_ad = heart.make_config(wl.B, wl.H, wl.N, wl.block, flags=heart.ESTIMATOR_ANTIDIAG)
+    ws_ad = heart.new_workspace(cfg_ad, dev)
+    ms_mask_ad_all = timed(lambda: heart.heart_predict_mask(cfg_ad, Q, Kt, tau, st_m, ws_ad), 3)
+    assert heart.heart_get_status(ws_ad) == 0
+    dens_ad = float(st_m.kv_cnt.to(torch.float64).mean()) / wl.n_blocks
+    groups = wl.N // 16
+    ad_flops = 2.0 * wl.R * float(groups) ** 2 * 16 * wl.D
+    ad_ws_bytes = ws_ad.numel()
+    del ws_ad, st_m
+
     hbm = stats_bytes / (ms_drift * 1e-3) / 1e9
     hbm_b2b = stats_bytes / (ms_drift_b2b * 1e-3) / 1e9
     l2_note = ("inputs larger than L2 (every step reads new Q/K/V tensors, >= 3x the 126 MB L2)"
@@ -337,6 +367,11 @@ def measure(torch, heart, inputs, replicas, wl, K, W, dev, pk, rank, sampler_uui
         "l2": l2_note,
         "stages_ms": {"drift": ms_drift, "mask": ms_mask, "attention": ms_attn,
                       "sum_of_separate_calls": ms_drift + ms_mask + ms_attn},
+        "mask_all_heads_ms": {"pooled": ms_mask_pooled_all, "strided_antidiagonal": ms_mask_ad_all,
+                              "pooled_density": dens_pooled, "strided_antidiagonal_density": dens_ad,
+                              "strided_antidiagonal_contraction_tflop": ad_flops / 1e12,
+                              "strided_antidiagonal_tflops_whole_call": ad_flops / (ms_mask_ad_all * 1e-3) / 1e12,
+                              "strided_antidiagonal_workspace_bytes": ad_ws_bytes},
         "density": density, "refresh_rate": refreshed / (K * wl.R),
         "retained_tflops": attn_tflops,
         "dense_equivalent_tflops": dense_flops / (ms_attn * 1e-3) / 1e12,
@@ -444,7 +479,7 @@ def run_ours(args, rank, world):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": rec["config"], "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": rec["l2"],
         }
-        for k in ("stages_ms", "density", "refresh_rate", "retained_tflops", "dense_equivalent_tflops",
+        for k in ("stages_ms", "mask_all_heads_ms", "density", "refresh_rate", "retained_tflops", "dense_equivalent_tflops",
                   "dense_equivalent_speedup_at_same_throughput", "attention_ms_back_to_back",
                   "retained_tflops_back_to_back", "dense_attention_ms_measured", "dense_tflops_measured",
                   "attention_speedup_vs_measured_dense", "roofline", "roofline_stats", "gpu_launches",
@@ -455,7 +490,7 @@ def run_ours(args, rank, world):
             out["cpu_baseline"] = cpu
         out["per_workload"] = [
             {"workload": r["workload"], "config": r["config"], "steps": r["steps"], "ms_per_step": r["ms_per_step"],
-             "stages_ms": r["stages_ms"], "density": r["density"], "refresh_rate": r["refresh_rate"],
+             "stages_ms": r["stages_ms"], "mask_all_heads_ms": r["mask_all_heads_ms"], "density": r["density"], "refresh_rate": r["refresh_rate"],
              "retained_tflops": r["retained_tflops"], "retained_tflops_back_to_back": r["retained_tflops_back_to_back"],
              "attention_frac": r["roofline"]["frac"], "attention_frac_of_burst_peak": r["roofline"]["frac_of_burst_peak"],
              "attention_frac_of_sustained_peak": r["roofline"]["frac_of_sustained_peak"],
