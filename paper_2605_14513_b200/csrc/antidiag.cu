@@ -78,7 +78,11 @@ __global__ void __launch_bounds__(kThreadsAd, 1)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int bidx = r / p.H, hidx = r % p.H;
   const int a0 = blockIdx.x * kMt;
-  const int n_tiles = (p.Ns + kNt - 1) / kNt;
+  // The key groups are dealt to gridDim.z CTAs per (row tile, head): every key block's pair is written
+  // by exactly one of them, so nothing has to be combined.  This CTA takes tiles [tile0, tile0 + n_tiles).
+  const int all_tiles = (p.Ns + kNt - 1) / kNt;
+  const int tile0 = (int)((long long)all_tiles * blockIdx.z / gridDim.z);
+  const int n_tiles = (int)((long long)all_tiles * (blockIdx.z + 1) / gridDim.z) - tile0;
   const int n_steps = n_tiles * kKSteps;
 
   if (tid == 0) {
@@ -121,7 +125,7 @@ __global__ void __launch_bounds__(kThreadsAd, 1)
         mbar_expect_tx(&bars->full[st], kStageBytes);
         // token t of the query groups a0 .. a0+127; token s-1-t of the key groups of this tile
         tma_load_5d(dst, &map_q, &bars->full[st], dh * 64, t, a0, hidx, bidx);
-        tma_load_5d(dst + kABytes, &map_k, &bars->full[st], dh * 64, kS - 1 - t, tile * kNt, hidx, bidx);
+        tma_load_5d(dst + kABytes, &map_k, &bars->full[st], dh * 64, kS - 1 - t, (tile0 + tile) * kNt, hidx, bidx);
         issued = it + 1;
       }
       if (*abort)  // shared memory must not be released under a copy in flight
@@ -177,7 +181,7 @@ __global__ void __launch_bounds__(kThreadsAd, 1)
       ok = __all_sync(0xffffffffu, mbar_wait(&bars->acc_full[buf], m & 1, abort));
       if (!ok) break;
       tc_fence_after();
-      const int c0 = tile * kNt;
+      const int c0 = (tile0 + tile) * kNt;
 #pragma unroll 1
       for (int ch = 0; ch < kNt / 32; ++ch) {
         if (c0 + ch * 32 >= p.Ns) break;  // (uniform) nothing but padding from here on
@@ -349,7 +353,22 @@ cudaError_t launch_antidiag_scores(const Geom &g, const Workspace &w, const void
     prm.g = grp;
     prm.c2 = (float)(g.scale / (double)kS * 1.4426950408889634);
     const int smem = kStagesAd * kStageBytes + 1024 + 256;
-    dim3 grid((Ns + kMt - 1) / kMt, g.R);
+    // Split the key range over up to four CTAs per (row tile, head) when that fills the 148 SMs' waves
+    // better (one CTA per SM); a shape-only rule.
+    const int row_tiles = (Ns + kMt - 1) / kMt, col_tiles = (Ns + kNt - 1) / kNt;
+    int split = 1;
+    double best_eff = 0.0;
+    for (int c = 1; c <= 4 && c <= col_tiles; ++c) {
+      const long long ctas = (long long)row_tiles * g.R * c;
+      const double waves = (double)((ctas + 147) / 148);
+      const int longest = (col_tiles + c - 1) / c;  // column tiles of the busiest CTA
+      const double eff = (double)ctas / (148.0 * waves) * ((double)col_tiles / c) / longest;
+      if (eff > best_eff + 0.02) {
+        best_eff = eff;
+        split = c;
+      }
+    }
+    dim3 grid(row_tiles, g.R, split);
     cudaError_t e;
     if (grp == 4) {
       e = cudaFuncSetAttribute(antidiag_scores_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
