@@ -246,15 +246,17 @@ __device__ __forceinline__ double exp_nonpos(double x) {
 // One CTA per (query block I, head r), fp64: the (max, sum) pairs of the block's groups become
 // scores[r][I][J] = ln(importance(I, J)) (-inf for importance 0), which the top-p kernel reads like
 // pooled scores.  A query block without a full group gets equal scores (uniform importance).
-// Reductions have a fixed shape (per-thread ascending, then a fixed tree): bit-reproducible.
-__global__ void __launch_bounds__(256) antidiag_reduce_kernel(const float2 *__restrict__ pairs, int Ns, int nb, int g,
-                                                              int pitch, const uint8_t *__restrict__ refresh,
-                                                              double *__restrict__ scores) {
+// One warp per group of the block (at most 8): row maximum and row sum by shuffles, the weights of
+// the lane's key blocks stay in registers in between; the groups are then added into the block's
+// weights one after the other.  Every reduction has a fixed shape: bit-reproducible.
+template <int NJ>  // NJ * 32 >= n_b
+__global__ void __launch_bounds__(256, 2) antidiag_reduce_kernel(const float2 *__restrict__ pairs, int Ns, int nb,
+                                                                 int g, int pitch, const uint8_t *__restrict__ refresh,
+                                                                 double *__restrict__ scores) {
   const int I = blockIdx.x, r = blockIdx.y;
   if (refresh != nullptr && refresh[r] == 0) return;
   __shared__ double wgt[HEART_MAX_BLOCKS];
-  __shared__ double red[256];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int a0 = I * g, a1 = min(a0 + g, Ns);
   const int nJ = (Ns + g - 1) / g;  // key blocks that hold at least one full group
   double *srow = scores + ((size_t)r * nb + I) * pitch;
@@ -263,36 +265,42 @@ __global__ void __launch_bounds__(256) antidiag_reduce_kernel(const float2 *__re
     return;
   }
   for (int J = tid; J < nb; J += 256) wgt[J] = 0.0;
+  constexpr int kPerLane = NJ;
   const double ln2 = 0.6931471805599453;
-  for (int a = a0; a < a1; ++a) {
+  double e[kPerLane];
+  double inv_z = 0.0;
+  const int a = a0 + warp;  // this warp's group (g <= 8 warps have one)
+  if (warp < g && a < a1) {
     const float2 *prow = pairs + ((size_t)r * Ns + a) * nb;
-    double mx = -INFINITY;
-    for (int J = tid; J < nJ; J += 256) mx = fmax(mx, (double)prow[J].x);
-    red[tid] = mx;
-    __syncthreads();
-    for (int w = 128; w > 0; w >>= 1) {
-      if (tid < w) red[tid] = fmax(red[tid], red[tid + w]);
-      __syncthreads();
-    }
-    mx = red[0];
-    __syncthreads();
+    float mxf = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < kPerLane; ++k)
+      if (lane + 32 * k < nJ) mxf = fmaxf(mxf, prow[lane + 32 * k].x);
+    double mx = (double)mxf;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     double z = 0.0;
-    for (int J = tid; J < nJ; J += 256) {
-      const float2 pr = prow[J];
-      z += exp_nonpos(((double)pr.x - mx) * ln2) * (double)pr.y;
+#pragma unroll
+    for (int k = 0; k < kPerLane; ++k) {
+      e[k] = 0.0;
+      if (lane + 32 * k < nJ) {  // (the row is in L1 / L2 from the pass above)
+        const float2 pr = prow[lane + 32 * k];
+        e[k] = exp_nonpos(((double)pr.x - mx) * ln2) * (double)pr.y;
+      }
+      z += e[k];
     }
-    red[tid] = z;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+    inv_z = 1.0 / z;
+  }
+  __syncthreads();
+  for (int aa = 0; aa < g; ++aa) {  // groups in ascending order: a fixed summation order
+    if (warp == aa && a < a1) {
+#pragma unroll
+      for (int k = 0; k < kPerLane; ++k)
+        if (lane + 32 * k < nJ) wgt[lane + 32 * k] += e[k] * inv_z;
+    }
     __syncthreads();
-    for (int w = 128; w > 0; w >>= 1) {
-      if (tid < w) red[tid] += red[tid + w];
-      __syncthreads();
-    }
-    z = red[0];
-    __syncthreads();
-    for (int J = tid; J < nJ; J += 256) {
-      const float2 pr = prow[J];
-      wgt[J] += exp_nonpos(((double)pr.x - mx) * ln2) * (double)pr.y / z;  // same thread owns J in every round
-    }
   }
   const double inv = 1.0 / (double)(a1 - a0);
   for (int J = tid; J < pitch; J += 256) {
@@ -382,8 +390,17 @@ cudaError_t launch_antidiag_scores(const Geom &g, const Workspace &w, const void
     ++*launches;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  antidiag_reduce_kernel<<<dim3(g.nb, g.R), 256, 0, s>>>(reinterpret_cast<const float2 *>(w.pairs), Ns, g.nb, grp,
-                                                          pitch, refresh, w.scores);
+  const float2 *pairs = reinterpret_cast<const float2 *>(w.pairs);
+  const dim3 rgrid(g.nb, g.R);
+  const int nj = (g.nb + 31) / 32;
+  if (nj <= 8)
+    antidiag_reduce_kernel<8><<<rgrid, 256, 0, s>>>(pairs, Ns, g.nb, grp, pitch, refresh, w.scores);
+  else if (nj <= 16)
+    antidiag_reduce_kernel<16><<<rgrid, 256, 0, s>>>(pairs, Ns, g.nb, grp, pitch, refresh, w.scores);
+  else if (nj <= 24)
+    antidiag_reduce_kernel<24><<<rgrid, 256, 0, s>>>(pairs, Ns, g.nb, grp, pitch, refresh, w.scores);
+  else
+    antidiag_reduce_kernel<32><<<rgrid, 256, 0, s>>>(pairs, Ns, g.nb, grp, pitch, refresh, w.scores);
   ++*launches;
   return cudaGetLastError();
 }
