@@ -157,6 +157,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
 #endif
 
   // ------------------------------------------------------------------ set-up
+  // A kernel that follows on the stream under programmatic stream serialisation (the next layer-step's
+  // block-sum pass) may be scheduled once every tile of this launch has started: its CTAs then fill the
+  // SMs that the last tiles leave behind and wait there for this launch to complete.
+  pdl_launch_dependents();
   if (tid == 0) HEART_TR(0, 28);
   // The lists of this tile's query blocks come from global memory: their loads are issued first
   // (speculatively, inside the row pitch) so that their latency overlaps the rest of the set-up.

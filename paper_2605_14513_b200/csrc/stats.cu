@@ -43,6 +43,13 @@ __global__ void __launch_bounds__(256, 5) block_sums_kernel(const uint16_t *__re
   const int i0 = chunk * bpc, i1 = min(nb, i0 + bpc);
   const int u0 = i0 * UPB, u1 = i1 * UPB;
   __shared__ float sm[2][16][kD];
+  // Launched with programmatic stream serialisation: when the kernel before it on the stream allows it
+  // (the library's own kernels do), these CTAs are scheduled while that kernel drains and wait here until
+  // it has completed and its writes are visible; after any other kernel this returns at once.
+  pdl_wait();
+  // The grid is one wave, so every CTA is past this point right after that: the follow-up kernel's CTAs
+  // are scheduled as soon as the first CTAs of this one leave, and wait there for the rest.
+  pdl_launch_dependents();
   if (chunk == 0 && r == 0 && z == 0 && threadIdx.x == 0) *sig_word = sig;  // whose means these are
 
   uint4 cur[ITERS], nxt[ITERS];
@@ -60,10 +67,7 @@ __global__ void __launch_bounds__(256, 5) block_sums_kernel(const uint16_t *__re
   double blk = 0.0;    // threads 0..127: sum of the current block so far
   int buf = 0;
   for (int u = u0; u < u1; ++u, buf ^= 1) {
-    if (u + 1 < u1)
-      load_unit(u + 1, nxt);
-    else
-      pdl_launch_dependents();  // the last loads of this CTA are on their way
+    if (u + 1 < u1) load_unit(u + 1, nxt);
     float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) {
@@ -253,12 +257,12 @@ cudaError_t launch_block_sums(const Geom &g, const void *Q, const void *K, const
   const uint16_t *q = static_cast<const uint16_t *>(Q), *k = static_cast<const uint16_t *>(K);
   unsigned long long *sig_word = reinterpret_cast<unsigned long long *>(w.status + kStatusSigWord);
   const unsigned long long sig = block_means_signature(g, Q, K);
-  if (g.block == 64)
-    block_sums_kernel<64><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bmean, w.psum, sig_word, sig);
-  else
-    block_sums_kernel<128><<<grid, 256, 0, s>>>(q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc, w.bmean, w.psum, sig_word, sig);
   ++*launches;
-  return cudaGetLastError();
+  if (g.block == 64)
+    return launch_pdl(block_sums_kernel<64>, grid, dim3(256), 0, s, q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc,
+                      w.bmean, w.psum, sig_word, sig);
+  return launch_pdl(block_sums_kernel<128>, grid, dim3(256), 0, s, q, k, g.sb, g.sh, g.sn, g.H, g.N, g.nb, g.bpc,
+                    w.bmean, w.psum, sig_word, sig);
 }
 
 cudaError_t launch_decide(const Geom &g, const Workspace &w, const double *delta, heart_state st,
