@@ -28,10 +28,13 @@
 // Tensor memory (256 columns per CTA): O | S[2]  =  128 + 2 x 64; key step h uses S[h & 1] and
 // shared-memory stage h & 1; P_h aliases S[h & 1].
 //
-// CTAs run head-major (the K/V of one or two heads stay in L2); the tiles of the last two heads of a
-// launch are taken longest-list-first from a table that tail_order_kernel writes just before, so that
-// the launch does not end on a long tile that started late.  The K tile of the first listed key block
-// is requested during set-up, before the step list is complete, and that block is put first.
+// CTAs run head-major (the K/V of one or two heads stay in L2).  Within a head the tiles are taken in
+// an order that tile_order_kernel writes just before the launch: by the first key block of their
+// lists, so that the ~300 tiles in flight together read neighbouring key blocks (a head's K and V no
+// longer fit one die's half of the L2 at 75 000 tokens and more), except for the last two heads of the
+// launch, whose tiles go longest-list-first so that the launch does not end on a long tile that
+// started late.  The K tile of the first listed key block is requested during set-up, before the step
+// list is complete, and that block is put first.
 //
 // Every wait is bounded; a wait that runs out raises a CTA-wide abort flag and the status word, the
 // roles drain, tensor memory is freed and the CTA exits.
@@ -91,8 +94,7 @@ struct AttnParams {
   long long sb, sh, sn;
   int H, N, nb, idx_stride, n_ctas_per_head, dense;
   int h0, hcount, R_all;  // this launch covers heads [h0, h0 + hcount) of every batch entry; R_all = B*H
-  const int32_t *order;   // the last n_sorted CTAs take their tile from this table (longest lists first)
-  int n_sorted;
+  const int32_t *order;   // [heads of the launch][n_ctas_per_head]: tile of the head that CTA i takes (NULL: i)
   float scale_log2;
   int test_skip_v;  // test-hook builds only: CTA 0 leaves out the V copy of its second key step
 };
@@ -137,15 +139,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
   // same role (above all the issuer of the score products) on the same sub-partition.
   const int kWarpKProd = 4 + ((kRoleKProd + blockIdx.x) & 3), kWarpVProd = 4 + ((kRoleVProd + blockIdx.x) & 3),
             kWarpPV = 4 + ((kRolePV + blockIdx.x) & 3), kWarpQK = 4 + ((kRoleQK + blockIdx.x) & 3);
-  // Tiles run head-major, which keeps the K/V of one or two heads in L2.  Only the tiles of the
-  // last two heads are taken longest-first from a table: the launch then ends on short tiles
-  // instead of waiting for a long one that started late.
-  int tile = blockIdx.x;
-  {
-    const int first_sorted = (int)gridDim.x - p.n_sorted;
-    if (tile >= first_sorted) tile = first_sorted + __ldg(&p.order[tile - first_sorted]);
-  }
-  const int rr = tile / p.n_ctas_per_head, cta_in_head = tile % p.n_ctas_per_head;
+  // Tiles run head-major, which keeps the K/V of one or two heads in L2; within a head in the order
+  // of the table (tiles whose lists start at the same key block together; the last two heads
+  // longest-first, so that the launch ends on short tiles).
+  const int rr = blockIdx.x / p.n_ctas_per_head;
+  const int cta_in_head = p.order ? __ldg(&p.order[blockIdx.x]) : (int)(blockIdx.x % p.n_ctas_per_head);
   const int bidx = rr / p.hcount, hidx = p.h0 + rr % p.hcount;
   const int r = bidx * p.H + hidx;
   const int row0 = cta_in_head * 128;  // first query token of this CTA
@@ -627,31 +625,36 @@ __global__ void __launch_bounds__(kAttnThreads, 2)
   if (tid == 0 && bars->abort) atomicExch(p.status, HEART_ERR_DEVICE_CHECK);
 }
 
-// Order of the last `n` tiles of a launch (those of its last one or two heads): descending by the
-// number of listed key blocks, ties by tile index -- rank by counting, so `order` is a permutation
-// whatever the counts hold.  n <= 2048.  Eight threads share a tile (each counts an eighth of the
-// keys), 32 tiles per CTA.
-__global__ void __launch_bounds__(256) tail_order_kernel(const int32_t *__restrict__ kv_cnt, int nb, int qbt, int ncph,
-                                                         int idx_stride, int H, int h0, int hcount, int rr0, int n,
-                                                         int32_t *__restrict__ order) {
-  __shared__ int key[2048];
-  for (int t = threadIdx.x; t < n; t += blockDim.x) {
-    const int rr = rr0 + t / ncph, r = (rr / hcount) * H + h0 + rr % hcount;
-    const int I0 = (t % ncph) * qbt;
-    int k = 0;
-    if (I0 < nb) k += min(max(__ldg(&kv_cnt[(size_t)r * nb + I0]), 0), idx_stride);
-    if (qbt == 2 && I0 + 1 < nb) k += min(max(__ldg(&kv_cnt[(size_t)r * nb + I0 + 1]), 0), idx_stride);
-    key[t] = k;
+// Order of the tiles of every head of a launch.  One CTA per head; rank by counting over at most 1024
+// keys, so the result is a permutation whatever the lists hold.  Heads before the last two: index order
+// while a head's K and V fit the L2 comfortably; beyond that ascending by the first key block that the
+// tile's lists name (ties by tile index) -- tiles that read the same region of K and V run together.
+// The last two heads: descending by the number of listed key blocks.
+__global__ void __launch_bounds__(256) tile_order_kernel(const int32_t *__restrict__ kv_idx,
+                                                         const int32_t *__restrict__ kv_cnt, int nb, int qbt, int ncph,
+                                                         int idx_stride, int H, int h0, int hcount, int n_heads,
+                                                         int by_first_key, int32_t *__restrict__ order) {
+  __shared__ int key[1024];
+  const int rr = blockIdx.x, r = (rr / hcount) * H + h0 + rr % hcount;
+  const bool by_length = rr >= n_heads - 2;
+  for (int t = threadIdx.x; t < ncph; t += blockDim.x) {
+    int len = 0, first = 0x3fffffff;
+    for (int qb = 0; qb < qbt; ++qb) {
+      const int I = t * qbt + qb;
+      if (I >= nb) break;
+      const int c = min(max(__ldg(&kv_cnt[(size_t)r * nb + I]), 0), idx_stride);
+      len += c;
+      if (c > 0) first = min(first, max(__ldg(&kv_idx[((size_t)r * nb + I) * idx_stride]), 0));
+    }
+    key[t] = by_length ? -len : (by_first_key ? first : t);
   }
   __syncthreads();
-  const int t = blockIdx.x * 32 + (threadIdx.x >> 3), part = threadIdx.x & 7;
-  const int mine = t < n ? key[t] : 0;
-  int rank = 0;
-  for (int u = part; u < n; u += 8) rank += (key[u] > mine || (key[u] == mine && u < t)) ? 1 : 0;
-  rank += __shfl_xor_sync(0xffffffffu, rank, 1);
-  rank += __shfl_xor_sync(0xffffffffu, rank, 2);
-  rank += __shfl_xor_sync(0xffffffffu, rank, 4);
-  if (part == 0 && t < n) order[rank] = t;
+  for (int t = threadIdx.x; t < ncph; t += blockDim.x) {
+    const int mine = key[t];
+    int rank = 0;
+    for (int u = 0; u < ncph; ++u) rank += (key[u] < mine || (key[u] == mine && u < t)) ? 1 : 0;
+    order[(size_t)rr * ncph + rank] = t;
+  }
 }
 
 // ---------------------------------------------------------------------- host side
@@ -732,22 +735,21 @@ cudaError_t launch_attention(const Geom &g, const void *Q, const void *K, const 
   prm.hcount = hcount;
   prm.R_all = g.R;
   prm.scale_log2 = (float)(g.scale * 1.4426950408889634);
-  prm.order = order;
   prm.test_skip_v = 0;
 #ifdef HEART_TEST_HOOKS
   prm.test_skip_v = (g.flags & 0x80000000u) ? 1 : 0;
 #endif
-  prm.n_sorted = 0;
-  if (!dense && order != nullptr) {
-    const int rows = g.B * hcount, nlast = rows < 2 ? rows : 2, n = nlast * prm.n_ctas_per_head;
-    if (n <= 2048) {
-      tail_order_kernel<<<(n + 31) / 32, 256, 0, s>>>(kv_cnt, g.nb, 128 / g.block, prm.n_ctas_per_head, g.idx_stride,
-                                                        g.H, h0, hcount, rows - nlast, n, order);
-      cudaError_t e = cudaGetLastError();
-      if (e != cudaSuccess) return e;
-      prm.n_sorted = n;
-      ++*launches;
-    }
+  prm.order = nullptr;
+  if (!dense && order != nullptr && prm.n_ctas_per_head <= 1024) {
+    const int rows = g.B * hcount;
+    // K + V of one head beyond 32 MB (about half of one die's share of the L2): order by key locality
+    const int by_first_key = (size_t)g.N * kD * 2 * 2 > (size_t)(32u << 20) ? 1 : 0;
+    tile_order_kernel<<<rows, 256, 0, s>>>(kv_idx, kv_cnt, g.nb, 128 / g.block, prm.n_ctas_per_head, g.idx_stride, g.H,
+                                           h0, hcount, rows, by_first_key, order);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    prm.order = order;
+    ++*launches;
   }
   ++*launches;
   return g.block == 64 ? launch_bk<64>(g, mq, mk, mv, prm, s) : launch_bk<128>(g, mq, mk, mv, prm, s);

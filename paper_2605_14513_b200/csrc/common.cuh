@@ -44,7 +44,7 @@ struct Workspace {
   uint8_t *pre;       // [R]            head-wise decision before the gate
   uint8_t *refresh;   // [R]            final decision of the current step
   double *drift;      // [R]
-  int32_t *order;     // [2048] tile order of the last two heads of an attention launch
+  int32_t *order;     // [R * ceil(N / 128)] order in which an attention launch takes the tiles of each head
   double *scores;     // [R][nb][pitch] pooled scores of the refreshed heads, pitch = nb rounded up to 32
   void *pairs;        // strided antidiagonal estimator only (HEART_ESTIMATOR_ANTIDIAG in the flags):
                       // float2 [R][N/16][nb], a (max, sum) pair per (query group, key block)
@@ -73,7 +73,7 @@ __host__ inline Workspace carve(const Geom &g, void *base) {
   w.drift = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * (size_t)g.R);
   w.order = reinterpret_cast<int32_t *>(p + off);
-  off += align256(sizeof(int32_t) * 2048);
+  off += align256(sizeof(int32_t) * (size_t)g.R * (size_t)((g.N + 127) / 128));
   w.bytes_drift = off;
   w.scores = reinterpret_cast<double *>(p + off);
   off += align256(sizeof(double) * (size_t)g.R * g.nb * (size_t)(((g.nb + 31) / 32) * 32));
