@@ -61,3 +61,11 @@ def test_reference_arm_prints_on_rank0_only():
     lines = [json.loads(l) for l in out.stdout.splitlines() if l.startswith("{")]
     assert len(lines) == 1 and lines[0]["impl"] == "reference" and lines[0]["n_gpus"] == 2
     assert lines[0]["cpu_baseline"]["kind"] == "oracle" and lines[0]["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_gpu_count_must_match_the_ranks_that_were_started():
+    """`--gpus N` inside a launch of another size is an error, not a silent single-replica run."""
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0")
+    out = subprocess.run([sys.executable, "bench.py", "--gpus", "2", "--workload", "tiny"], capture_output=True,
+                         text=True, env=env, cwd=ROOT, timeout=120)
+    assert out.returncode == 2 and "WORLD_SIZE" in out.stderr
