@@ -217,32 +217,6 @@ __global__ void __launch_bounds__(kThreadsAd, 1)
   if (tid == 0 && bars->abort) atomicExch(p.status, HEART_ERR_DEVICE_CHECK);
 }
 
-// exp(x) for x <= 0 (same construction as in the top-p kernel: magic-number rint, two-step
-// reduction, degree-13 Taylor, exponent add); 0 below -708.
-__device__ __forceinline__ double exp_nonpos(double x) {
-  if (!(x >= -708.0)) return 0.0;
-  const double t = fma(x, 1.4426950408889634, 6755399441055744.0);
-  const int n = __double2loint(t);
-  const double fn = t - 6755399441055744.0;
-  double r = fma(fn, -6.93147180369123816490e-01, x);
-  r = fma(fn, -1.90821492927058770002e-10, r);
-  double q = 1.6059043836821613e-10;
-  q = fma(q, r, 2.08767569878681e-09);
-  q = fma(q, r, 2.505210838544172e-08);
-  q = fma(q, r, 2.755731922398589e-07);
-  q = fma(q, r, 2.7557319223985893e-06);
-  q = fma(q, r, 2.48015873015873e-05);
-  q = fma(q, r, 1.984126984126984e-04);
-  q = fma(q, r, 1.388888888888889e-03);
-  q = fma(q, r, 8.333333333333333e-03);
-  q = fma(q, r, 4.1666666666666664e-02);
-  q = fma(q, r, 1.6666666666666666e-01);
-  q = fma(q, r, 0.5);
-  q = fma(q, r, 1.0);
-  q = fma(q, r, 1.0);
-  return __hiloint2double(__double2hiint(q) + (n << 20), __double2loint(q));
-}
-
 // One CTA per (query block I, head r), fp64: the (max, sum) pairs of the block's groups become
 // scores[r][I][J] = ln(importance(I, J)) (-inf for importance 0), which the top-p kernel reads like
 // pooled scores.  A query block without a full group gets equal scores (uniform importance).
@@ -285,7 +259,7 @@ __global__ void __launch_bounds__(256, 2) antidiag_reduce_kernel(const float2 *_
       e[k] = 0.0;
       if (lane + 32 * k < nJ) {  // (the row is in L1 / L2 from the pass above)
         const float2 pr = prow[lane + 32 * k];
-        e[k] = exp_nonpos(((double)pr.x - mx) * ln2) * (double)pr.y;
+        e[k] = exp_nonpositive(((double)pr.x - mx) * ln2) * (double)pr.y;
       }
       z += e[k];
     }
@@ -309,26 +283,10 @@ __global__ void __launch_bounds__(256, 2) antidiag_reduce_kernel(const float2 *_
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void *sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(sym);
-  }();
-  return fn;
-}
-
 // bf16 [B,H,N,128] seen as (dim, token in group, group, head, batch); box = 64 dims of one token
 // position of `rows` consecutive groups, 128-byte swizzle, groups past Ns read as zero.
 bool make_group_map(CUtensorMap *m, const void *base, const Geom &g, int Ns, int rows) {
-  EncodeTiledFn fn = encode_fn();
+  EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[5] = {(cuuint64_t)kD, (cuuint64_t)kS, (cuuint64_t)Ns, (cuuint64_t)g.H, (cuuint64_t)g.B};
   cuuint64_t strides[4] = {(cuuint64_t)g.sn * 2, (cuuint64_t)g.sn * 2 * kS, (cuuint64_t)g.sh * 2, (cuuint64_t)g.sb * 2};

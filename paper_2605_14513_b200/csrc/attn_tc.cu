@@ -660,26 +660,10 @@ __global__ void __launch_bounds__(256) tile_order_kernel(const int32_t *__restri
 // ---------------------------------------------------------------------- host side
 namespace {
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = []() -> EncodeTiledFn {
-    void *sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      return nullptr;
-    return reinterpret_cast<EncodeTiledFn>(sym);
-  }();
-  return fn;
-}
-
 // bf16 [B,H,N,128] with element strides (sb, sh, sn, 1): box = 64 dims x `rows` tokens, 128-byte swizzle,
 // out-of-range rows read as zero.
 bool make_map(CUtensorMap *m, const void *base, const Geom &g, int rows) {
-  EncodeTiledFn fn = encode_fn();
+  EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)g.N, (cuuint64_t)g.H, (cuuint64_t)g.B};
   cuuint64_t strides[3] = {(cuuint64_t)g.sn * 2, (cuuint64_t)g.sh * 2, (cuuint64_t)g.sb * 2};

@@ -37,35 +37,6 @@ __device__ __forceinline__ double warp_max(double v) {
   return v;
 }
 
-// exp(x) for x <= 0 in about a third of the instructions of the library routine, which spends most of
-// its time on ranges that cannot occur here: n = rint(x log2 e) by the magic-number add, r = x - n ln 2
-// in two steps, the Taylor polynomial of degree 13 on |r| <= ln 2 / 2 (truncation 4e-18), 2^n by an
-// integer add into the exponent field.  Below -708 (weights under 1e-307 of the row maximum) it
-// returns 0.  Within an ulp or two of the correctly rounded value, like the library routine.
-__device__ __forceinline__ double exp_nonpositive(double x) {
-  if (x < -708.0) return 0.0;
-  const double t = fma(x, 1.4426950408889634, 6755399441055744.0);
-  const int n = __double2loint(t);
-  const double fn = t - 6755399441055744.0;
-  double r = fma(fn, -6.93147180369123816490e-01, x);
-  r = fma(fn, -1.90821492927058770002e-10, r);
-  double q = 1.6059043836821613e-10;            // 1/13!
-  q = fma(q, r, 2.08767569878681e-09);          // 1/12!
-  q = fma(q, r, 2.505210838544172e-08);         // 1/11!
-  q = fma(q, r, 2.755731922398589e-07);         // 1/10!
-  q = fma(q, r, 2.7557319223985893e-06);        // 1/9!
-  q = fma(q, r, 2.48015873015873e-05);          // 1/8!
-  q = fma(q, r, 1.984126984126984e-04);         // 1/7!
-  q = fma(q, r, 1.388888888888889e-03);         // 1/6!
-  q = fma(q, r, 8.333333333333333e-03);         // 1/5!
-  q = fma(q, r, 4.1666666666666664e-02);        // 1/4!
-  q = fma(q, r, 1.6666666666666666e-01);        // 1/3!
-  q = fma(q, r, 0.5);
-  q = fma(q, r, 1.0);
-  q = fma(q, r, 1.0);
-  return __hiloint2double(__double2hiint(q) + (n << 20), __double2loint(q));
-}
-
 // 8-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros instead
 __device__ __forceinline__ void cp_async8(double *smem_dst, const double *src, int src_bytes) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)),

@@ -105,3 +105,47 @@ def test_full_size_shapes_on_sampled_rows(heart, oracle, name, n_sample):
     print(f"[{name}] antidiagonal estimator: {differing} of {len(picks)} sampled rows differ inside the bands; "
           f"density {cnt.mean() / nb:.3f}")
     assert differing <= max(1, n_sample // 16)
+
+
+def test_strided_layout_and_padded_index_pitch(heart, oracle):
+    """Q and K stored [B, N, H, D] and viewed as [B, H, N, D]: the estimator's 5-D tensor maps take
+    the strides from the config; the index lists get a padded row pitch."""
+    rs = np.random.RandomState(23)
+    B, H, N, D, b = 2, 3, 700, 128, 64   # 43 full groups + 12 unsampled tokens
+    nb = (N + b - 1) // b
+    store = [(torch.randn(B, N, H, D, device="cuda") * 1.5).to(torch.bfloat16) for _ in range(2)]
+    Q, K = (s.permute(0, 2, 1, 3) for s in store)
+    cfg = heart.config_for(Q, b, idx_stride=nb + 3, flags=heart.ESTIMATOR_ANTIDIAG)
+    st, ws = heart.State(cfg), heart.new_workspace(cfg)
+    tau_np = rs.uniform(0.5, 0.95, B * H)
+    tau = torch.tensor(tau_np, dtype=torch.float64, device="cuda")
+    heart.heart_predict_mask(cfg, Q, K, tau, st, ws)
+    assert heart.heart_get_status(ws) == 0
+    Qb, Kb = (inputs.bits(t.contiguous()) for t in (Q, K))
+    ost = oracle.State(B, H, N, D, b, idx_stride=nb + 3)
+    oracle.predict_mask_antidiag(Qb, Kb, b, tau_np, ost)
+    assert check_masks(st, ost, range(B * H), tau_np, lambda r, I: oracle.antidiag_probs_row(Qb, Kb, b, r, I)) <= 1
+
+
+def test_host_buffer_step_with_this_estimator(heart, oracle):
+    """heart_step_host honours the flag: identical masks, flags and output to heart_step."""
+    wl = inputs.small_workload(H=3, grid=(3, 10, 14), block=128, seed=29, steps=2, eps=[0.01, 0.1, 0.3],
+                               delta=[0.6, 0.6, 0.6])
+    a, b = antidiag_pair(wl, heart, oracle), antidiag_pair(wl, heart, oracle)
+    staging = tuple(torch.empty_like(b.Q) for _ in range(4))
+    for t in range(2):
+        O = torch.full_like(a.Q, float("nan"))
+        r1 = torch.empty(wl.R, dtype=torch.uint8, device="cuda")
+        heart.heart_step(a.cfg, a.Q, a.K, a.V, a.delta, a.tau, a.gst, O, a.ws, refresh_out=r1)
+        host = [x.cpu().contiguous().pin_memory() for x in (b.Q, b.K, b.V)]
+        Oh = torch.full(b.Q.shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+        rh = torch.full((wl.R,), 7, dtype=torch.uint8).pin_memory()
+        heart.heart_step_host(b.cfg, host[0], host[1], host[2], b.delta, b.tau, b.gst, Oh, staging, b.ws, refresh_host=rh)
+        torch.cuda.current_stream().synchronize()
+        assert heart.heart_get_status(a.ws) == 0 and heart.heart_get_status(b.ws) == 0
+        assert np.array_equal(to_np(r1), rh.numpy())
+        assert torch.equal(O.cpu().view(torch.int16), Oh.view(torch.int16))
+        for x, y in zip(a.gst.tensors(), b.gst.tensors()):
+            assert torch.equal(x, y)
+        a.advance()
+        b.advance()
