@@ -352,7 +352,7 @@ def test_state_reset(heart, oracle):
 
 # ------------------------------------------------------------------ the benchmark configurations
 @pytest.mark.parametrize("name,steps,n_sample", [
-    ("wan1.3b-480p", 3, 64),
+    ("wan1.3b-480p", 8, 64),   # eight steps: heads that never, sometimes and always refresh
     ("wan14b-480p", 2, 64),
     ("wan14b-720p", 2, 64),
     ("hunyuan-720p", 2, 64),
