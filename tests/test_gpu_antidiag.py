@@ -149,3 +149,22 @@ def test_host_buffer_step_with_this_estimator(heart, oracle):
             assert torch.equal(x, y)
         a.advance()
         b.advance()
+
+
+def test_maximum_block_count_with_this_estimator(heart, oracle):
+    """n_b = 1024 at block 64 (4095 groups, 16 column tiles dealt to several CTAs per row tile): sampled rows."""
+    wl = inputs.small_workload(H=1, grid=(1, 1, 64 * 1024 - 9), block=64, seed=13, tau=[0.9])
+    assert wl.n_blocks == heart.MAX_BLOCKS
+    p = antidiag_pair(wl, heart, oracle)
+    heart.heart_predict_mask(p.cfg, p.Q, p.K, p.tau, p.gst, p.ws)
+    assert heart.heart_get_status(p.ws) == 0
+    cnt, idx = to_np(p.gst.kv_cnt), to_np(p.gst.kv_idx)
+    differing = 0
+    for I in (0, 1, 255, 256, 511, 777, 1022, 1023):
+        P = oracle.antidiag_probs_row(p.Qb, p.Kb, wl.block, 0, I)
+        keep, k, _, _ = oracle.top_p(P, 0.9)
+        G, Rf = set(idx[0, I, :cnt[0, I]].tolist()), set(np.nonzero(keep)[0].tolist())
+        if G != Rf:
+            check_differing_row(G, Rf, P, 0.9, wl.n_blocks, (0, I))
+            differing += 1
+    assert differing <= 1
